@@ -1,0 +1,471 @@
+// hs_accept_path: two launches.
+//
+// accept_rows_kernel   vocabulary pass over the target row of every kept node (arg-max with lowest
+//                      index on ties; for sampling sequences also max and sum e^((x-max)/T)) and
+//                      over the draft row of every kept internal node of a sampling sequence.
+//                      Same register-resident 16-byte-load pattern as the entropy pass; the last
+//                      chunk of a row merges the chunk partials.
+// accept_walk_kernel   one thread-block cluster per sequence walks the tree from the root.
+//                      Greedy (temperature 0): follow the child whose token is the arg-max.
+//                      Sampling (Sec. 2.1): test siblings in index order with u < min(1, r/q); the
+//                      residual after k rejections is max(p - c_k q, 0) / W_k with c_0 = 0, W_0 = 1,
+//                      c_(k+1) = c_k + W_k, W_k = sum_v max(p_v - c_k q_v, 0), so a rejection costs
+//                      one vocabulary-wide sum, split over the CTAs of the cluster and exchanged
+//                      through distributed shared memory.  The bonus token is drawn by inverse CDF
+//                      in token order.
+#include <cooperative_groups.h>
+#include <math_constants.h>
+
+#include "hs_common.cuh"
+#include "hs_layout.h"
+
+namespace cg = cooperative_groups;
+
+#define LOG2E 1.4426950408889634f
+#define WALK_CLUSTER 8
+#define WALK_THREADS 512
+
+struct RowOut {           // per kept node, in the workspace
+    int* tgt_arg;         // arg-max token of the target row
+    float2* tgt_ms;       // {max, sum e^((x-max)/T)} of the target row
+    float2* drf_ms;       // same for the draft row (internal nodes of sampling sequences)
+};
+
+struct AcceptParams {
+    const void* target;
+    const void* draft;
+    int64_t row_stride;
+    int vocab, nvec, chunks, chunk_vecs, is_bf16;
+    int batch, n_nodes_total, target_layout;
+    const int* node_off;
+    const int* token;
+    hs_pruned_tree pr;
+    const int* mode;
+    const float* temperature;
+    unsigned long long seed, offset;
+    const float* uniforms;
+    hs_accept_out out;
+    RowOut ro;
+    uint4* partials;      // [2][max_rows][chunks] {key lo, key hi, max, sum}
+    int* row_cnt;
+};
+
+__device__ __forceinline__ float ex2a(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+template <bool BF16>
+__device__ __forceinline__ void unpack_v(const uint4& v, float* x) {
+    if (BF16) {
+        x[0] = bf16_lo(v.x); x[1] = bf16_hi(v.x); x[2] = bf16_lo(v.y); x[3] = bf16_hi(v.y);
+        x[4] = bf16_lo(v.z); x[5] = bf16_hi(v.z); x[6] = bf16_lo(v.w); x[7] = bf16_hi(v.w);
+    } else {
+        x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y);
+        x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
+    }
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(HS_ROW_THREADS, 2) accept_rows_kernel(const AcceptParams p) {
+    constexpr int VE = BF16 ? 8 : 4;
+    constexpr int VPT = HS_ROW_VPT;
+    __shared__ float s_w[8][2];
+    __shared__ unsigned long long s_key[8];
+    __shared__ int s_flag;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int chunk = blockIdx.x, k = blockIdx.y, which = blockIdx.z;   // which: 0 target, 1 draft
+    if (k >= p.pr.keep_off[p.batch]) return;
+    int lo = 0, hi = p.batch;                     // sequence of kept node k
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (p.pr.keep_off[mid] <= k) lo = mid; else hi = mid;
+    }
+    const int b = lo;
+    const int i = k - p.pr.keep_off[b];
+    const int nk = p.pr.n_keep[b];
+    const bool sampling = p.mode[b] == HS_ACCEPT_REJECTION;
+    if (which == 1) {
+        if (!sampling) return;
+        int internal = 0;                         // does kept node i have a kept child?
+        for (int j = i + 1 + tid; j < nk; j += HS_ROW_THREADS)
+            internal |= (p.pr.new_parent[p.pr.keep_off[b] + j] == i);
+        if (!__syncthreads_or(internal)) return;
+    }
+    const int orig_row = p.node_off[b] + p.pr.keep_idx[k];
+    const int row = which == 1 ? orig_row : (p.target_layout == HS_ROWS_ORIGINAL ? orig_row : k);
+    const char* rowp = (const char*)(which == 1 ? p.draft : p.target) + (size_t)row * p.row_stride * (BF16 ? 2 : 4);
+    const int v0 = chunk * p.chunk_vecs;
+    const int v1 = min(v0 + p.chunk_vecs, p.nvec);
+
+    uint4 d[VPT];
+#pragma unroll
+    for (int j = 0; j < VPT; ++j) {
+        int v = v0 + tid + j * HS_ROW_THREADS;
+        if (v < v1) {
+            d[j] = __ldcs((const uint4*)(rowp) + v);
+        } else {
+            unsigned int ninf = BF16 ? 0xff80ff80u : 0xff800000u;
+            d[j] = make_uint4(ninf, ninf, ninf, ninf);
+        }
+    }
+    // per-thread best (value, lowest index)
+    float tmax = -CUDART_INF_F;
+    int targ = 0x7fffffff;
+#pragma unroll
+    for (int j = 0; j < VPT; ++j) {
+        float x[8];
+        unpack_v<BF16>(d[j], x);
+        int base = (v0 + tid + j * HS_ROW_THREADS) * VE;
+#pragma unroll
+        for (int e = 0; e < VE; ++e) {
+            bool in = base + e < p.vocab;
+            if (in && x[e] > tmax) { tmax = x[e]; targ = base + e; }   // ascending index: strict > keeps the lowest
+        }
+    }
+    unsigned long long key = (targ == 0x7fffffff) ? 0ull : make_key(tmax, targ);
+    key = warp_max_u64(key);
+    float s = 0.f;
+    if (sampling) {
+        const float invT = LOG2E / p.temperature[b];
+        const float nml = (tmax == -CUDART_INF_F) ? 0.f : -tmax * invT;
+#pragma unroll
+        for (int j = 0; j < VPT; ++j) {
+            float x[8];
+            unpack_v<BF16>(d[j], x);
+            int base = (v0 + tid + j * HS_ROW_THREADS) * VE;
+#pragma unroll
+            for (int e = 0; e < VE; ++e)
+                if (base + e < p.vocab) s += ex2a(fmaf(fmaxf(x[e], -1e30f), invT, nml));
+        }
+        float wm = warp_max(tmax);
+        float f = (tmax == -CUDART_INF_F) ? 0.f : ex2a((tmax - wm) * invT);
+        s = warp_sum(s * f);
+        if (lane == 0) { s_w[warp][0] = wm; s_w[warp][1] = s; }
+    }
+    if (lane == 0) s_key[warp] = key;
+    __syncthreads();
+    if (tid == 0) {
+        unsigned long long best = s_key[0];
+        for (int w = 1; w < 8; ++w) best = s_key[w] > best ? s_key[w] : best;
+        float M = -CUDART_INF_F, S = 0.f;
+        if (sampling) {
+            const float invT = LOG2E / p.temperature[b];
+            for (int w = 0; w < 8; ++w) M = fmaxf(M, s_w[w][0]);
+            for (int w = 0; w < 8; ++w)
+                S += (s_w[w][0] == -CUDART_INF_F) ? 0.f : s_w[w][1] * ex2a((s_w[w][0] - M) * invT);
+        }
+        p.partials[((size_t)which * HS_MAX_ROWS + k) * p.chunks + chunk] =
+            make_uint4((unsigned int)best, (unsigned int)(best >> 32), __float_as_uint(M), __float_as_uint(S));
+        __threadfence();
+        int* cnt = &p.row_cnt[which * HS_MAX_ROWS + k];
+        s_flag = (atomicAdd(cnt, 1) == p.chunks - 1);
+        if (s_flag) *cnt = 0;
+    }
+    __syncthreads();
+    if (!s_flag || warp != 0) return;
+    __threadfence();
+    // last chunk of the row: merge (chunks <= 32, one lane per chunk)
+    unsigned long long ck = 0ull;
+    float cm = -CUDART_INF_F, cs = 0.f;
+    if (lane < p.chunks) {
+        uint4 q = __ldcg(&p.partials[((size_t)which * HS_MAX_ROWS + k) * p.chunks + lane]);
+        ck = ((unsigned long long)q.y << 32) | q.x;
+        cm = __uint_as_float(q.z);
+        cs = __uint_as_float(q.w);
+    }
+    unsigned long long best = warp_max_u64(ck);
+    float M = warp_max(cm), S = 0.f;
+    if (sampling) {
+        const float invT = LOG2E / p.temperature[b];
+        S = warp_sum((cm == -CUDART_INF_F) ? 0.f : cs * ex2a((cm - M) * invT));
+    }
+    if (lane == 0) {
+        if (which == 0) {
+            p.ro.tgt_arg[k] = key_index(best);
+            p.ro.tgt_ms[k] = make_float2(M, S);
+        } else {
+            p.ro.drf_ms[k] = make_float2(M, S);
+        }
+    }
+}
+
+// ---- the walk ----------------------------------------------------------------------------------
+
+__device__ __forceinline__ float load_logit(const void* base, int is_bf16, size_t off) {
+    return is_bf16 ? __bfloat162float(((const __nv_bfloat16*)base)[off]) : ((const float*)base)[off];
+}
+
+// Sum over this CTA's share of the vocabulary of max(p_v - c q_v, 0), then over the cluster.
+// Every CTA returns the same value (fixed summation order).
+__device__ double cluster_residual_sum(const AcceptParams& p, cg::cluster_group& cluster, const char* prow,
+                                       const char* qrow, float pm, float ips, float qm, float iqs, float invT,
+                                       float c, double* s_part, double* s_cta) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int ve = p.is_bf16 ? 8 : 4;
+    const unsigned int rank = cluster.block_rank();
+    const int per = (p.nvec + WALK_CLUSTER - 1) / WALK_CLUSTER;
+    const int v0 = rank * per, v1 = min(v0 + per, p.nvec);
+    float acc = 0.f;
+    for (int v = v0 + tid; v < v1; v += WALK_THREADS) {
+        uint4 a = __ldg((const uint4*)prow + v), bq = __ldg((const uint4*)qrow + v);
+        float x[8], y[8];
+        if (p.is_bf16) { unpack_v<true>(a, x); unpack_v<true>(bq, y); }
+        else { unpack_v<false>(a, x); unpack_v<false>(bq, y); }
+        for (int e = 0; e < ve; ++e) {
+            if (v * ve + e < p.vocab) {
+                float pv = ex2a((fmaxf(x[e], -1e30f) - pm) * invT) * ips;
+                float qv = ex2a((fmaxf(y[e], -1e30f) - qm) * invT) * iqs;
+                acc += fmaxf(pv - c * qv, 0.f);
+            }
+        }
+    }
+    double w = warp_sum_d((double)acc);
+    if (lane == 0) s_part[warp] = w;
+    __syncthreads();
+    if (tid == 0) {
+        double t = 0.0;
+        for (int i = 0; i < WALK_THREADS / 32; ++i) t += s_part[i];
+        *s_cta = t;
+    }
+    cluster.sync();
+    double tot = 0.0;
+    for (unsigned int r = 0; r < WALK_CLUSTER; ++r) tot += *cluster.map_shared_rank(s_cta, r);
+    cluster.sync();                     // nobody overwrites s_cta before all have read it
+    return tot;
+}
+
+// Inverse-CDF draw from max(p - c q, 0) in token order: smallest j whose running sum exceeds
+// u * total; if rounding leaves none, the last token with positive mass.  `qrow` may be NULL (c = 0).
+__device__ int cluster_inverse_cdf(const AcceptParams& p, cg::cluster_group& cluster, const char* prow,
+                                   const char* qrow, float pm, float ips, float qm, float iqs, float invT,
+                                   float c, float u, double* s_scan, double* s_cta, int* s_pick) {
+    const int tid = threadIdx.x;
+    const unsigned int rank = cluster.block_rank();
+    const int per_cta = (p.vocab + WALK_CLUSTER - 1) / WALK_CLUSTER;
+    const int c0 = rank * per_cta, c1 = min(c0 + per_cta, p.vocab);
+    const int seg = (per_cta + WALK_THREADS - 1) / WALK_THREADS;
+    const int t0 = min(c0 + tid * seg, c1), t1 = min(t0 + seg, c1);
+    auto mass = [&](int j) -> float {
+        float pv = ex2a((fmaxf(load_logit(prow, p.is_bf16, j), -1e30f) - pm) * invT) * ips;
+        if (qrow == nullptr) return pv;
+        float qv = ex2a((fmaxf(load_logit(qrow, p.is_bf16, j), -1e30f) - qm) * invT) * iqs;
+        return fmaxf(pv - c * qv, 0.f);
+    };
+    double mine = 0.0;
+    int last_pos = -1;
+    for (int j = t0; j < t1; ++j) {
+        float r = mass(j);
+        mine += (double)r;
+        if (r > 0.f) last_pos = j;
+    }
+    s_scan[tid] = mine;
+    if (tid == 0) { s_pick[0] = 0x7fffffff; s_pick[1] = -1; }
+    __syncthreads();
+    if (tid == 0) {                       // serial exclusive scan over the CTA's threads (512 adds)
+        double run = 0.0;
+        for (int i = 0; i < WALK_THREADS; ++i) { double v = s_scan[i]; s_scan[i] = run; run += v; }
+        *s_cta = run;
+    }
+    cluster.sync();
+    double before = 0.0, total = 0.0;
+    for (unsigned int r = 0; r < WALK_CLUSTER; ++r) {
+        double v = *cluster.map_shared_rank(s_cta, r);
+        if (r < rank) before += v;
+        total += v;
+    }
+    const double goal = (double)u * total;
+    double run = before + s_scan[tid];
+    if (run <= goal && run + mine > goal) {          // the crossing lies in this thread's segment
+        for (int j = t0; j < t1; ++j) {
+            run += (double)mass(j);
+            if (run > goal) { atomicMin(&s_pick[0], j); break; }
+        }
+    }
+    if (last_pos >= 0) atomicMax(&s_pick[1], last_pos);
+    __syncthreads();
+    cluster.sync();
+    int pick = 0x7fffffff, lastp = -1;
+    for (unsigned int r = 0; r < WALK_CLUSTER; ++r) {
+        const int* sp = cluster.map_shared_rank(s_pick, r);
+        pick = min(pick, sp[0]);
+        lastp = max(lastp, sp[1]);
+    }
+    cluster.sync();
+    return pick != 0x7fffffff ? pick : max(lastp, 0);
+}
+
+__global__ void __cluster_dims__(WALK_CLUSTER, 1, 1) __launch_bounds__(WALK_THREADS)
+accept_walk_kernel(const AcceptParams p) {
+    cg::cluster_group cluster = cg::this_cluster();
+    __shared__ double s_part[WALK_THREADS / 32];
+    __shared__ double s_scan[WALK_THREADS];
+    __shared__ double s_cta;
+    __shared__ int s_pick[2];
+    __shared__ int s_child;
+    const int tid = threadIdx.x;
+    const int b = blockIdx.x / WALK_CLUSTER;
+    const unsigned int rank = cluster.block_rank();
+    const int koff = p.pr.keep_off[b];
+    const int nk = p.pr.n_keep[b];
+    const int nbase = p.node_off[b];
+    const int cap = p.out.path_cap;
+    const bool sampling = p.mode[b] == HS_ACCEPT_REJECTION;
+    const size_t esz = p.is_bf16 ? 2 : 4;
+
+    if (rank == 0) {
+        for (int j = tid; j < cap; j += WALK_THREADS) {
+            p.out.path_nodes[b * cap + j] = -1;
+            p.out.path_compact[b * cap + j] = -1;
+            p.out.path_tokens[b * cap + j] = -1;
+        }
+    }
+    if (nk <= 0 || p.pr.status[b] != 0) {
+        if (rank == 0 && tid == 0) {
+            p.out.accept_len[b] = 0; p.out.bonus_token[b] = -1; p.out.terminal_rank[b] = -1;
+            p.out.status[b] = p.pr.status[b] != 0 ? p.pr.status[b] : HS_ERR_BAD_TREE;
+        }
+        return;
+    }
+    __syncthreads();
+    int cur = 0, len = 0, bonus = -1;
+    if (!sampling) {
+        if (rank != 0) return;
+        for (int step = 0; step < nk; ++step) {
+            const int g = p.ro.tgt_arg[koff + cur];
+            if (tid == 0) s_child = 0x7fffffff;
+            __syncthreads();
+            for (int j = cur + 1 + tid; j < nk; j += WALK_THREADS)
+                if (p.pr.new_parent[koff + j] == cur && p.token[nbase + p.pr.keep_idx[koff + j]] == g)
+                    atomicMin(&s_child, j);
+            __syncthreads();
+            const int nxt = s_child;
+            __syncthreads();
+            if (tid == 0 && len < cap) {
+                p.out.path_compact[b * cap + len] = cur;
+                p.out.path_nodes[b * cap + len] = p.pr.keep_idx[koff + cur];
+            }
+            if (nxt == 0x7fffffff) { bonus = g; break; }
+            if (tid == 0 && len < cap) p.out.path_tokens[b * cap + len] = g;
+            cur = nxt;
+            ++len;
+        }
+    } else {
+        const float T = p.temperature[b];
+        const float invT = LOG2E / T;
+        for (int step = 0; step < nk; ++step) {
+            if (rank == 0 && tid == 0 && len < cap) {
+                p.out.path_compact[b * cap + len] = cur;
+                p.out.path_nodes[b * cap + len] = p.pr.keep_idx[koff + cur];
+            }
+            const int trow = p.target_layout == HS_ROWS_ORIGINAL ? nbase + p.pr.keep_idx[koff + cur] : koff + cur;
+            const int drow = nbase + p.pr.keep_idx[koff + cur];
+            const char* prow = (const char*)p.target + (size_t)trow * p.row_stride * esz;
+            const char* qrow = (const char*)p.draft + (size_t)drow * p.row_stride * esz;
+            const float2 pms = p.ro.tgt_ms[koff + cur];
+            const float pm = pms.x, ips = 1.f / pms.y;
+            float qm = 0.f, iqs = 0.f;
+            bool have_q = false;
+            float c = 0.f;
+            double W = 1.0;
+            int accepted = -1;
+            bool tested = false;
+            for (int j = cur + 1; j < nk; ++j) {                 // siblings in index order
+                if (p.pr.new_parent[koff + j] != cur) continue;
+                if (!have_q) {
+                    const float2 qms = p.ro.drf_ms[koff + cur];
+                    qm = qms.x; iqs = 1.f / qms.y; have_q = true;
+                }
+                tested = true;
+                const int orig = p.pr.keep_idx[koff + j];
+                const int t = p.token[nbase + orig];
+                const float pt = ex2a((fmaxf(load_logit(prow, p.is_bf16, t), -1e30f) - pm) * invT) * ips;
+                const float qt = ex2a((fmaxf(load_logit(qrow, p.is_bf16, t), -1e30f) - qm) * invT) * iqs;
+                const float r = fmaxf(pt - c * qt, 0.f) / (float)W;
+                const float a = qt > 0.f ? fminf(1.f, r / qt) : 1.f;
+                const float u = p.uniforms ? p.uniforms[nbase + orig] : philox_uniform(p.seed, p.offset, b, orig, 0);
+                if (u < a) { accepted = j; break; }
+                const float c_next = c + (float)W;
+                const double W_next = cluster_residual_sum(p, cluster, prow, qrow, pm, ips, qm, iqs, invT,
+                                                           c_next, s_part, &s_cta);
+                if (!(W_next > 0.0)) { c = 0.f; W = 1.0; tested = false; break; }   // p == q: fall back to p
+                c = c_next; W = W_next;
+            }
+            if (accepted >= 0) {
+                if (rank == 0 && tid == 0 && len < cap)
+                    p.out.path_tokens[b * cap + len] = p.token[nbase + p.pr.keep_idx[koff + accepted]];
+                cur = accepted;
+                ++len;
+                continue;
+            }
+            const float ufin = p.uniforms ? p.uniforms[p.n_nodes_total + b] : philox_uniform(p.seed, p.offset, b, 0, 1);
+            bonus = cluster_inverse_cdf(p, cluster, prow, (tested && c > 0.f) ? qrow : nullptr, pm, ips, qm, iqs,
+                                        invT, c, ufin, s_scan, &s_cta, s_pick);
+            break;
+        }
+    }
+    if (rank == 0 && tid == 0) {
+        p.out.accept_len[b] = len;
+        p.out.bonus_token[b] = bonus;
+        p.out.terminal_rank[b] = p.pr.keep_rank[koff + cur];
+        p.out.status[b] = HS_OK;
+    }
+}
+
+__global__ void philox_kernel(unsigned long long seed, unsigned long long offset, const int* b, const int* node,
+                              const int* stream_id, int count, float* out) {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < count) out[i] = philox_uniform(seed, offset, b[i], node[i], stream_id[i]);
+}
+
+hs_status hs_launch_philox(uint64_t seed, uint64_t offset, const int32_t* b, const int32_t* node,
+                           const int32_t* stream_id, int32_t count, float* out, cudaStream_t stream) {
+    philox_kernel<<<(count + 255) / 256, 256, 0, stream>>>(seed, offset, b, node, stream_id, count, out);
+    return cudaGetLastError() == cudaSuccess ? HS_OK : HS_ERR_CUDA;
+}
+
+hs_status hs_launch_accept(hs_ctx* ctx, const hs_tree_batch* tree, const hs_pruned_tree* pruned,
+                           const void* target_logits, int32_t target_layout, const void* draft_logits,
+                           hs_dtype dtype, int64_t row_stride, int32_t vocab, const int32_t* mode,
+                           const float* temperature, uint64_t seed, uint64_t offset, const float* uniforms,
+                           const hs_accept_out* out, cudaStream_t stream) {
+    AcceptParams p;
+    const int ve = hs_vec_elems(dtype);
+    p.target = target_logits;
+    p.draft = draft_logits ? draft_logits : target_logits;   // only read by sampling sequences
+    p.row_stride = row_stride;
+    p.vocab = vocab;
+    p.nvec = (vocab + ve - 1) / ve;
+    p.chunks = hs_row_chunks(vocab, dtype);
+    if (p.chunks > 32) return HS_ERR_SHAPE;
+    p.chunk_vecs = (p.nvec + p.chunks - 1) / p.chunks;
+    p.is_bf16 = dtype == HS_BF16;
+    p.batch = tree->batch;
+    p.n_nodes_total = tree->n_nodes_total;
+    p.target_layout = target_layout;
+    p.node_off = tree->node_off;
+    p.token = tree->token;
+    p.pr = *pruned;
+    p.mode = mode;
+    p.temperature = temperature;
+    p.seed = seed;
+    p.offset = offset;
+    p.uniforms = uniforms;
+    p.out = *out;
+    const int rows = tree->n_nodes_total;          // upper bound of kept nodes
+    size_t o = 0;
+    p.ro.tgt_arg = (int*)(ctx->scratch + o); o += hs_align_up((size_t)rows * sizeof(int), 256);
+    p.ro.tgt_ms = (float2*)(ctx->scratch + o); o += hs_align_up((size_t)rows * sizeof(float2), 256);
+    p.ro.drf_ms = (float2*)(ctx->scratch + o); o += hs_align_up((size_t)rows * sizeof(float2), 256);
+    p.partials = (uint4*)(ctx->scratch + o);
+    o += (size_t)(HS_MAX_ROWS + rows) * p.chunks * sizeof(uint4);
+    if (o > ctx->scratch_bytes) return HS_ERR_WORKSPACE;
+    p.row_cnt = ctx->counters + HS_CNT_ACC_ROW;
+    dim3 grid(p.chunks, rows, 2);
+    if (dtype == HS_BF16) accept_rows_kernel<true><<<grid, HS_ROW_THREADS, 0, stream>>>(p);
+    else accept_rows_kernel<false><<<grid, HS_ROW_THREADS, 0, stream>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return HS_ERR_CUDA;
+    accept_walk_kernel<<<p.batch * WALK_CLUSTER, WALK_THREADS, 0, stream>>>(p);
+    return cudaGetLastError() == cudaSuccess ? HS_OK : HS_ERR_CUDA;
+}

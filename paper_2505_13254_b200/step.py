@@ -1,0 +1,103 @@
+"""One verification step on the GPU: uploads a synthetic batch and chains the four C-ABI calls.
+
+Only plumbing lives here (device buffers, the order of the calls); every step of the path runs
+inside the CUDA library.
+"""
+
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+import torch
+
+from . import binding as hb
+
+
+def _bf16(bits: np.ndarray, device) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(device).view(torch.bfloat16)
+
+
+def _logits(x: np.ndarray, device) -> torch.Tensor:
+    return _bf16(x, device) if x.dtype == np.uint16 else torch.from_numpy(np.ascontiguousarray(x)).to(device)
+
+
+@dataclass
+class DeviceBatch:
+    """A batch as the input generators emit it, resident on the device.  Rows of the logits and of
+    q / k_tree / v_tree are indexed by drafted node id (HS_ROWS_ORIGINAL)."""
+    tree: hb.TreeBatch
+    draft: Optional[torch.Tensor]
+    target: Optional[torch.Tensor]
+    q: Optional[torch.Tensor]
+    k_tree: Optional[torch.Tensor]
+    v_tree: Optional[torch.Tensor]
+    k_cache: Optional[torch.Tensor]
+    v_cache: Optional[torch.Tensor]
+    kv_off: torch.Tensor
+    mode: torch.Tensor
+    temperature: torch.Tensor
+    seed: int
+    offset: int
+    max_nodes: int
+    max_kv_len: int
+
+    def nbytes(self) -> int:
+        ts = [self.tree.node_off, self.tree.parent, self.tree.token, self.draft, self.target, self.q, self.k_tree,
+              self.v_tree, self.k_cache, self.v_cache, self.kv_off, self.mode, self.temperature]
+        return sum(t.numel() * t.element_size() for t in ts if t is not None)
+
+
+def upload(batch: dict, device="cuda:0") -> DeviceBatch:
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
+    node_off = np.asarray(batch["node_off"])
+    kv_off = np.asarray(batch["kv_off"])
+    tree = hb.TreeBatch(i32(node_off), i32(batch["parent"]), i32(batch["token"]), len(node_off) - 1, int(node_off[-1]))
+    get = lambda k, f: f(batch[k], device) if k in batch else None
+    return DeviceBatch(tree, get("draft", _logits), get("target", _logits), get("q", _bf16), get("k_tree", _bf16),
+                       get("v_tree", _bf16), get("k_cache", _bf16), get("v_cache", _bf16), i32(kv_off),
+                       i32(batch["mode"]),
+                       torch.from_numpy(np.asarray(batch["temperature"], dtype=np.float32)).to(device),
+                       int(batch["philox_seed"]), int(batch["philox_offset"]),
+                       int(np.diff(node_off).max()), int(np.diff(kv_off).max()))
+
+
+class VerifyStep:
+    """Pre-allocated outputs + the four calls in the order of the decode loop."""
+
+    def __init__(self, ctx: hb.Context, db: DeviceBatch, policy: dict, path_cap: int = 32):
+        dev = db.tree.parent.device
+        self.ctx, self.policy = ctx, policy
+        n, b = db.tree.n_nodes_total, db.tree.batch
+        self.quant = hb.QuantOut(n, b, policy["top_k"], dev)
+        self.pruned = hb.PrunedTree(n, b, dev)
+        self.accept = hb.AcceptOut(b, path_cap, dev)
+        self.attn_out = torch.zeros_like(db.q) if db.q is not None else None
+        self.attn_lse = (torch.zeros(db.q.shape[0], db.q.shape[1], dtype=torch.float32, device=dev)
+                         if db.q is not None else None)
+
+    def quantify(self, db: DeviceBatch):
+        return hb.hs_entropy_quantify(self.ctx, db.tree, db.draft, self.policy, out=self.quant)
+
+    def prune(self, db: DeviceBatch):
+        return hb.hs_stratify_prune(self.ctx, db.tree, self.quant, self.policy, out=self.pruned)
+
+    def attention(self, db: DeviceBatch):
+        return hb.hs_tree_verify_attention(self.ctx, self.pruned, db.q, db.k_tree, db.v_tree, db.k_cache, db.v_cache,
+                                           db.kv_off, batch=db.tree.batch, max_nodes=db.max_nodes,
+                                           max_kv_len=db.max_kv_len, layout=hb.HS_ROWS_ORIGINAL,
+                                           node_off=db.tree.node_off, out=self.attn_out, lse_out=self.attn_lse)
+
+    def accept_path(self, db: DeviceBatch):
+        return hb.hs_accept_path(self.ctx, db.tree, self.pruned, db.target, db.draft, db.mode, db.temperature,
+                                 target_layout=hb.HS_ROWS_ORIGINAL, seed=db.seed, offset=db.offset,
+                                 path_cap=self.accept.path_cap, out=self.accept)
+
+    def run(self, db: DeviceBatch):
+        self.quantify(db)
+        self.prune(db)
+        if db.q is not None:
+            self.attention(db)
+        self.accept_path(db)
+        return self

@@ -1,0 +1,143 @@
+"""Shared helpers of the GPU parity tests: guard-banded cases and element-wise comparisons."""
+import json
+import os
+
+import numpy as np
+
+from oracle import step as ostep
+from oracle import tree as otree
+from paper_2505_13254_b200 import synth
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+THRESHOLDS = json.load(open(os.path.join(GOLD, "thresholds.json")))
+
+# guard bands of the float -> integer decisions (the GPU decides in fp32, the oracle in fp64)
+BAND_BIN, BAND_RANK, BAND_PSTAR, BAND_ACCEPT, BAND_CDF = 1e-3, 1e-4, 1e-4, 1e-4, 1e-5
+
+
+def policy_for(cfg, base=None):
+    name = base or cfg.name
+    return synth.default_policy(cfg, THRESHOLDS[name]["thresholds"])
+
+
+def oracle_case(cfg, policy, seed, attention="full", attn_pairs=64, max_tries=20):
+    """Generates a batch whose every float decision keeps its guard band (else the next seed is
+    taken) and runs the oracle on it.  attention: "full" | "sampled" | "none"."""
+    for s in range(seed, seed + max_tries):
+        batch = synth.make_batch(cfg, s, with_attention=attention != "none")
+        res, ok = [], True
+        for b in range(cfg.batch):
+            stats, sc = ostep.quantify(batch, policy, b)
+            m = otree.margins(sc, policy)
+            if m["bin"] <= BAND_BIN or m["rank"] <= BAND_RANK or m["pstar"] <= BAND_PSTAR:
+                ok = False
+                break
+            pr = ostep.stratify_prune(batch, policy, b, sc)
+            trace = []
+            acc = ostep.accept_path(batch, b, pr, trace=trace)
+            for t in trace:
+                if t[0] == "accept" and abs(t[2] - t[3]) <= BAND_ACCEPT:
+                    ok = False
+                if t[0] == "final" and (t[1] - t[2] <= BAND_CDF or t[3] - t[1] <= BAND_CDF):
+                    ok = False
+            if not ok:
+                break
+            res.append(dict(stats=stats, scores=sc, pruned=pr, accept=acc))
+        if not ok:
+            continue
+        if attention != "none":
+            rng = np.random.default_rng(s)
+            for b, r in enumerate(res):
+                nk = len(r["pruned"]["keep_idx"])
+                pairs = None
+                if attention == "sampled":
+                    pairs = [(int(rng.integers(nk)), int(rng.integers(cfg.hq))) for _ in range(attn_pairs)]
+                    pairs += [(nk - 1, h) for h in range(0, cfg.hq, max(1, cfg.hq // 8))]
+                r["attn_out"], r["attn_lse"] = ostep.verify_attention(batch, b, r["pruned"], rows=pairs)
+        return batch, res
+    raise RuntimeError("no guard-banded seed found")
+
+
+def rel_close(got, want, rel=1e-4, abs_=1e-6):
+    got, want = np.asarray(got, dtype=np.float64), np.asarray(want, dtype=np.float64)
+    return np.all(np.abs(got - want) <= rel * np.abs(want) + abs_), float(np.max(np.abs(got - want) / (np.abs(want) + abs_ / rel)))
+
+
+def check_quant(q, batch, res, K):
+    """Entropies within 1e-4 relative; maxima, Top-K ids and values, depths and P* exact."""
+    node_off = batch["node_off"]
+    for b, r in enumerate(res):
+        lo, hi = node_off[b], node_off[b + 1]
+        st = r["stats"]
+        assert np.array_equal(q.row_max[lo:hi].cpu().numpy().astype(np.float64), [s["max"] for s in st])
+        for name, key in (("row_lse", "lse"), ("h_full", "H"), ("i_topk", "I_topk"), ("i_trunc", "I_trunc")):
+            ok, err = rel_close(getattr(q, name)[lo:hi].cpu().numpy(), [s[key] for s in st])
+            assert ok, (name, b, err)
+        assert np.array_equal(q.topk_idx[lo:hi].cpu().numpy(), np.stack([s["topk_idx"] for s in st]))
+        assert np.array_equal(q.topk_val[lo:hi].cpu().numpy().astype(np.float64), np.stack([s["topk_val"] for s in st]))
+        sc = r["scores"]
+        for name, key in (("logc", "logc"), ("score", "S"), ("phi", "Phi")):
+            ok, err = rel_close(getattr(q, name)[lo:hi].cpu().numpy(), sc[key], abs_=1e-5)
+            assert ok, (name, b, err)
+        assert np.array_equal(q.depth[lo:hi].cpu().numpy(), sc["depth"])
+        assert int(q.pstar_node[b]) == sc["pstar_node"]
+        ok, err = rel_close(float(q.phi_star[b]), sc["phi_star"], abs_=1e-5)
+        assert ok, ("phi_star", b, err)
+        assert int(q.status[b]) == 0
+
+
+def check_pruned(p, res):
+    """Bit-exact: bins, d', N', kept node sets, parents, depths, ranks and ancestor masks."""
+    off = p.keep_off.cpu().numpy()
+    for b, r in enumerate(res):
+        pr = r["pruned"]
+        nk = len(pr["keep_idx"])
+        assert (int(p.bin[b]), int(p.d_prime[b]), int(p.n_prime[b]), int(p.n_keep[b])) == \
+            (pr["bin"], pr["d_prime"], pr["n_prime"], nk)
+        assert off[b + 1] - off[b] == nk
+        sl = slice(off[b], off[b + 1])
+        assert np.array_equal(p.keep_idx[sl].cpu().numpy(), pr["keep_idx"])
+        assert np.array_equal(p.new_parent[sl].cpu().numpy(), pr["new_parent"])
+        assert np.array_equal(p.new_depth[sl].cpu().numpy(), pr["new_depth"])
+        assert np.array_equal(p.keep_rank[sl].cpu().numpy(), pr["rank"])
+        words = p.anc_mask[sl].cpu().numpy().view(np.uint64)
+        want = np.zeros((nk, 2), dtype=np.uint64)
+        for i in range(nk):
+            for j in np.nonzero(pr["mask"][i])[0]:
+                want[i, j // 64] |= np.uint64(1) << np.uint64(j % 64)
+        assert np.array_equal(words, want)
+
+
+def check_accept(a, res):
+    """Bit-exact: accepted length, path (original and compact ids), tokens, bonus token, rank."""
+    for b, r in enumerate(res):
+        acc = r["accept"]
+        n = acc["accept_len"]
+        assert int(a.status[b]) == 0
+        assert int(a.accept_len[b]) == n, (b, int(a.accept_len[b]), n)
+        assert a.path_nodes[b, : n + 1].tolist() == acc["path_nodes"]
+        assert a.path_compact[b, : n + 1].tolist() == acc["path_compact"]
+        assert a.path_tokens[b, :n].tolist() == acc["path_tokens"]
+        assert (a.path_nodes[b, n + 1:] == -1).all() and (a.path_tokens[b, n:] == -1).all()
+        assert int(a.bonus_token[b]) == acc["bonus"], (b, int(a.bonus_token[b]), acc["bonus"])
+        assert int(a.terminal_rank[b]) == acc["terminal_rank"]
+
+
+def check_attention(out, lse, batch, res, tol=1e-2):
+    """bf16 output of the kernels against the fp64 oracle: max absolute error <= tol on every
+    (node, head) the oracle evaluated; rows are laid out by drafted node id."""
+    node_off = batch["node_off"]
+    worst = 0.0
+    o = out.float().cpu().numpy().astype(np.float64)
+    l = lse.cpu().numpy().astype(np.float64)
+    for b, r in enumerate(res):
+        rows = node_off[b] + r["pruned"]["keep_idx"]
+        want, want_lse = r["attn_out"], r["attn_lse"]
+        got, got_lse = o[rows], l[rows]
+        done = ~np.isnan(want[..., 0])
+        assert done.any()
+        err = np.abs(got[done] - want[done]).max()
+        worst = max(worst, err)
+        assert err <= tol, (b, err)
+        assert np.abs(got_lse[done] - want_lse[done]).max() <= 1e-3 * max(1.0, np.abs(want_lse[done]).max())
+    return worst
