@@ -1,0 +1,301 @@
+#!/usr/bin/env python
+"""Benchmark of one HeteroSpec verification step (quantify -> stratify/prune -> tree attention ->
+accept) on synthetic inputs shaped like the Llama-3.1-8B workload.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload c2_8b]
+
+Prints ONE JSON line.  A "step" is one pass of the whole path over one batch; inputs rotate through
+several distinct device copies whose total size exceeds the L2 cache, so every step reads HBM.
+With N > 1 (torchrun) every rank verifies its own batch (independent trees: no collective on the
+data path) and the slowest rank's time is used.  `--impl reference` times the CPU oracle instead.
+"""
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "verified_draft_trees_per_second"
+UNIT = "trees/s"
+L2_BYTES = 126 << 20
+
+
+def load_policy(cfg, synth):
+    th = json.load(open(os.path.join(ROOT, "tests", "golden", "thresholds.json")))
+    return synth.default_policy(cfg, th[cfg.name]["thresholds"])
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons sampled while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.Q}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        rows = [r.strip().split(", ") for r in open(self.f.name) if r.strip()]
+        os.unlink(self.f.name)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.strip().lower() == "active":
+                    reasons.add(n)
+        if sm:
+            out = {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                   "samples": len(sm)}
+        return out
+
+
+def oracle_sample(batch, policy, ostep):
+    """One tree through the whole oracle path (all rows, all attention pairs of the kept nodes)."""
+    t = time.perf_counter()
+    ostep.verify_step(batch, policy, with_attention=True)
+    return time.perf_counter() - t
+
+
+def run_reference(args, cfg, synth):
+    from oracle import step as ostep
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    policy = load_policy(cfg, synth)
+    batch = synth.make_batch(cfg, 0)
+    times = []
+    for i in range(args.warmup + args.steps):
+        dt = oracle_sample(batch, policy, ostep)
+        if i >= args.warmup:
+            times.append(dt)
+    total = sum(times)
+    value = cfg.batch * len(times) / total
+    cores = os.cpu_count()
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": cfg.name, "batch": cfg.batch, "vocab": cfg.vocab,
+                                            "kv_len": cfg.kv_len[1], "hq": cfg.hq, "hkv": cfg.hkv},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": "each step = the whole batch through the numpy fp64 oracle (all logits rows, "
+                                       "all kept-node attention pairs of one layer); numpy/BLAS threads as configured"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2_8b")
+    ap.add_argument("--rotate", type=int, default=0, help="distinct input copies (0 = enough to exceed 2x L2)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    from paper_2505_13254_b200 import synth
+    cfg = synth.CONFIGS[args.workload]
+    if args.impl == "reference":
+        if args.steps > 20:
+            args.steps = 5                 # bounded: a step is seconds of CPU work
+            args.warmup = min(args.warmup, 1)
+        return run_reference(args, cfg, synth)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2505_13254_b200 import binding as hb
+    from paper_2505_13254_b200 import step as gstep
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the verification path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    policy = load_policy(cfg, synth)
+    batch = synth.make_batch(cfg, rank)                      # each rank verifies its own trees
+    db0 = gstep.upload(batch, dev)
+    per_set = db0.nbytes()
+    R = args.rotate or max(2, -(-2 * L2_BYTES // per_set) + 1)
+    sets = [db0]
+    for _ in range(R - 1):
+        c = gstep.upload(batch, dev)
+        sets.append(c)
+    ws = hb.hs_workspace_bytes(cfg.batch, db0.tree.n_nodes_total, cfg.vocab, cfg.hq, cfg.hkv)
+    ctx = hb.Context(local, ws)
+    st = gstep.VerifyStep(ctx, db0, policy)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing ----------------------------------------------------------------------
+    for i in range(args.warmup):
+        st.run(sets[i % R])
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        st.run(sets[i % R])
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    # ---- per-call durations (second pass over the same steps, events around every call) ----------------
+    calls = ("quantify", "prune", "attention", "accept_path")
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(calls) + 1)] for _ in range(args.steps)]
+    for i in range(args.steps):
+        db = sets[i % R]
+        evs[i][0].record()
+        for j, c in enumerate(calls):
+            getattr(st, c)(db)
+            evs[i][j + 1].record()
+    barrier()
+    call_us = {c: 1e3 * sum(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(args.steps)) / args.steps
+               for j, c in enumerate(calls)}
+    clocks = sampler.stop() if sampler else None
+    nk = int(st.pruned.n_keep.sum().item())
+    n_rows = db0.tree.n_nodes_total
+
+    # ---- end to end: pinned host inputs -> device, the four calls, results -> host, every step -----------
+    host = {}
+    names = ("draft", "target", "q", "k_tree", "v_tree", "k_cache", "v_cache")
+    for n in names:
+        host[n] = getattr(db0, n).cpu().pin_memory()
+    for n in ("node_off", "parent", "token"):
+        host[n] = getattr(db0.tree, n).cpu().pin_memory()
+    res_host = {n: getattr(st.accept, n).cpu().pin_memory() for n in ("accept_len", "path_tokens", "bonus_token")}
+    stage = sets[-1]
+    h2d = sum(t.numel() * t.element_size() for t in host.values())
+    d2h = sum(t.numel() * t.element_size() for t in res_host.values())
+
+    def e2e_step():
+        for n in names:
+            getattr(stage, n).copy_(host[n], non_blocking=True)
+        for n in ("node_off", "parent", "token"):
+            getattr(stage.tree, n).copy_(host[n], non_blocking=True)
+        st.run(stage)
+        for n, t in res_host.items():
+            t.copy_(getattr(st.accept, n), non_blocking=True)
+        torch.cuda.synchronize()
+
+    e2e_steps = min(args.steps, 100)
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e2e_s = time.perf_counter() - t0
+    barrier()
+
+    if world > 1:
+        t = torch.tensor([ms, e2e_s], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_s = float(t[0]), float(t[1])
+    dev_err = hb.hs_device_error(ctx)
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peaks()
+    esz = 2 if cfg.logits_dtype == "bf16" else 4
+    quant_bytes = n_rows * cfg.vocab * esz
+    L = int(np.diff(batch["kv_off"]).sum())
+    attn_bytes = 2 * (L + nk) * cfg.hkv * cfg.head_dim * 2 + 2 * nk * cfg.hq * cfg.head_dim * 2
+    accept_bytes = nk * cfg.vocab * esz
+    kern = {
+        "quantify": {"bytes": quant_bytes, "us": call_us["quantify"], "launches_per_step": 1},
+        "attention": {"bytes": attn_bytes, "us": call_us["attention"], "launches_per_step": 2},
+        "accept_path": {"bytes": accept_bytes, "us": call_us["accept_path"], "launches_per_step": 2},
+        "prune": {"bytes": 0, "us": call_us["prune"], "launches_per_step": 1},
+    }
+    for k in kern.values():
+        k["gbs"] = k["bytes"] / (k["us"] * 1e-6) / 1e9 if k["us"] > 0 else None
+        k["frac_of_%s_hbm" % peak_kind] = k["gbs"] / peak if k["gbs"] else None
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tpath):
+        traffic = json.load(open(tpath)).get(cfg.name, {}).get("quantify_kernel")
+    achieved = kern["quantify"]["gbs"]
+    line = {
+        "metric": METRIC, "value": world * cfg.batch * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": cfg.name, "batch_per_gpu": cfg.batch, "tree_nodes": n_rows, "kept_nodes": nk,
+                   "vocab": cfg.vocab, "logits_dtype": cfg.logits_dtype, "kv_len": cfg.kv_len[1], "hq": cfg.hq,
+                   "hkv": cfg.hkv, "head_dim": cfg.head_dim, "attention_layers_per_step": 1,
+                   "accept": cfg.accept, "parallelism": "replicas" if world > 1 else "single",
+                   "l2": "inputs rotate through %d distinct device copies, %.0f MB in total (L2 = 126 MB)"
+                         % (R, R * per_set / 1e6)},
+        "clocks": clocks,
+        "e2e": {"value": world * cfg.batch * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": 1e3 * e2e_s / e2e_steps},
+        "gpu_launches": 6 * args.steps,
+        "roofline": {"kernel": "quantify_kernel (hs_entropy_quantify, one launch per step)", "bound": "hbm",
+                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": peak_kind + " (burst copy figure)", "traffic": traffic,
+                     "algorithmic_bytes_per_launch": quant_bytes,
+                     "how": "CUDA events around every call in a second pass over the same steps"},
+        "calls": kern,
+        "device_error_word": dev_err,
+    }
+    if not args.no_cpu_baseline:
+        from oracle import step as ostep
+        t = oracle_sample(batch, policy, ostep)
+        line["cpu_baseline"] = {"value": cfg.batch / t, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+                                "sample": "the same batch once through the numpy fp64 oracle: all logits rows, "
+                                          "all kept-node attention pairs of one layer (%.1f s)" % t}
+    print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

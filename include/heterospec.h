@@ -75,6 +75,10 @@ size_t hs_workspace_bytes(int32_t max_batch, int32_t max_rows, int32_t vocab, in
 hs_status hs_create(hs_ctx** ctx, int32_t device, size_t workspace_bytes);
 hs_status hs_destroy(hs_ctx* ctx);
 
+/* Reads and clears the context's sticky device error word into *host_out (host pointer): HS_OK, or
+ * HS_ERR_TIMEOUT if a kernel gave up a bounded wait since the last call.  Synchronises the device. */
+hs_status hs_device_error(hs_ctx* ctx, int32_t* host_out);
+
 /* ---- descriptors -------------------------------------------------------------------------- */
 
 typedef struct {

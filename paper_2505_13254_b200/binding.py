@@ -59,7 +59,7 @@ class _AcceptOut(C.Structure):
                                   "terminal_rank", "status")] + [("path_cap", C.c_int32)]
 
 
-EXPORTS = ("hs_status_string", "hs_workspace_bytes", "hs_create", "hs_destroy", "hs_entropy_quantify",
+EXPORTS = ("hs_status_string", "hs_workspace_bytes", "hs_create", "hs_destroy", "hs_device_error", "hs_entropy_quantify",
            "hs_stratify_prune", "hs_tree_verify_attention", "hs_accept_path", "hs_philox_uniforms")
 
 
@@ -76,6 +76,7 @@ def lib() -> C.CDLL:
         L.hs_workspace_bytes.argtypes = [C.c_int32] * 5
         L.hs_create.argtypes = [C.POINTER(C.c_void_p), C.c_int32, C.c_size_t]
         L.hs_destroy.argtypes = [C.c_void_p]
+        L.hs_device_error.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
         L.hs_entropy_quantify.argtypes = [C.c_void_p, C.POINTER(_TreeBatch), vp, C.c_int, C.c_int64, C.c_int32,
                                           C.POINTER(_Policy), C.POINTER(_QuantOut), vp]
         L.hs_stratify_prune.argtypes = [C.c_void_p, C.POINTER(_TreeBatch), C.POINTER(_QuantOut),
@@ -110,6 +111,12 @@ def _ptr(t: Optional[torch.Tensor]):
 
 def _stream():
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def hs_device_error(ctx: "Context") -> int:
+    v = C.c_int32(0)
+    _check(lib().hs_device_error(ctx.handle, C.byref(v)), "hs_device_error")
+    return int(v.value)
 
 
 def hs_workspace_bytes(max_batch: int, max_rows: int, vocab: int, hq: int, hkv: int) -> int:

@@ -215,8 +215,8 @@ __device__ double cluster_residual_sum(const AcceptParams& p, cg::cluster_group&
         else { unpack_v<false>(a, x); unpack_v<false>(bq, y); }
         for (int e = 0; e < ve; ++e) {
             if (v * ve + e < p.vocab) {
-                float pv = ex2a((fmaxf(x[e], -1e30f) - pm) * invT) * ips;
-                float qv = ex2a((fmaxf(y[e], -1e30f) - qm) * invT) * iqs;
+                float pv = exp2f((fmaxf(x[e], -1e30f) - pm) * invT) * ips;
+                float qv = exp2f((fmaxf(y[e], -1e30f) - qm) * invT) * iqs;
                 acc += fmaxf(pv - c * qv, 0.f);
             }
         }
@@ -248,9 +248,9 @@ __device__ int cluster_inverse_cdf(const AcceptParams& p, cg::cluster_group& clu
     const int seg = (per_cta + WALK_THREADS - 1) / WALK_THREADS;
     const int t0 = min(c0 + tid * seg, c1), t1 = min(t0 + seg, c1);
     auto mass = [&](int j) -> float {
-        float pv = ex2a((fmaxf(load_logit(prow, p.is_bf16, j), -1e30f) - pm) * invT) * ips;
+        float pv = exp2f((fmaxf(load_logit(prow, p.is_bf16, j), -1e30f) - pm) * invT) * ips;
         if (qrow == nullptr) return pv;
-        float qv = ex2a((fmaxf(load_logit(qrow, p.is_bf16, j), -1e30f) - qm) * invT) * iqs;
+        float qv = exp2f((fmaxf(load_logit(qrow, p.is_bf16, j), -1e30f) - qm) * invT) * iqs;
         return fmaxf(pv - c * qv, 0.f);
     };
     double mine = 0.0;
@@ -380,8 +380,8 @@ accept_walk_kernel(const AcceptParams p) {
                 tested = true;
                 const int orig = p.pr.keep_idx[koff + j];
                 const int t = p.token[nbase + orig];
-                const float pt = ex2a((fmaxf(load_logit(prow, p.is_bf16, t), -1e30f) - pm) * invT) * ips;
-                const float qt = ex2a((fmaxf(load_logit(qrow, p.is_bf16, t), -1e30f) - qm) * invT) * iqs;
+                const float pt = exp2f((fmaxf(load_logit(prow, p.is_bf16, t), -1e30f) - pm) * invT) * ips;
+                const float qt = exp2f((fmaxf(load_logit(qrow, p.is_bf16, t), -1e30f) - qm) * invT) * iqs;
                 const float r = fmaxf(pt - c * qt, 0.f) / (float)W;
                 const float a = qt > 0.f ? fminf(1.f, r / qt) : 1.f;
                 const float u = p.uniforms ? p.uniforms[nbase + orig] : philox_uniform(p.seed, p.offset, b, orig, 0);

@@ -75,6 +75,17 @@ extern "C" hs_status hs_destroy(hs_ctx* ctx) {
     return HS_OK;
 }
 
+extern "C" hs_status hs_device_error(hs_ctx* ctx, int32_t* host_out) {
+    if (!ctx || !host_out) return HS_ERR_INVALID_ARG;
+    HS_CUDA_OK(cudaSetDevice(ctx->device));
+    HS_CUDA_OK(cudaDeviceSynchronize());
+    int v = 0;
+    HS_CUDA_OK(cudaMemcpy(&v, ctx->counters + HS_CNT_ERROR, sizeof(int), cudaMemcpyDeviceToHost));
+    if (v != 0) HS_CUDA_OK(cudaMemset(ctx->counters + HS_CNT_ERROR, 0, sizeof(int)));
+    *host_out = v;
+    return HS_OK;
+}
+
 static bool tree_ok(const hs_tree_batch* t) {
     return t && t->batch >= 1 && t->batch <= HS_MAX_BATCH && t->n_nodes_total >= t->batch &&
            t->n_nodes_total <= HS_MAX_ROWS && t->node_off && t->parent && t->token;

@@ -292,18 +292,25 @@ def make_sequence(cfg: VerifyConfig, seed: int, b: int, with_logits: bool = True
     return out
 
 
+SALT_STRIDE = 1_000_003
+
+
 def make_batch(cfg: VerifyConfig, seed: int, with_logits: bool = True,
-               with_attention: bool = True) -> dict:
+               with_attention: bool = True, salts=None) -> dict:
     """A ragged batch in CSR form.  Logits and Q/K/V of tree nodes are laid out by original
     node index (row ``node_off[b] + i`` belongs to node i of sequence b).  Logits are float32
-    values for ``logits_dtype == "f32"`` and uint16 bfloat16 bit patterns otherwise."""
-    seqs = [make_sequence(cfg, seed, b, with_logits, with_attention) for b in range(cfg.batch)]
+    values for ``logits_dtype == "f32"`` and uint16 bfloat16 bit patterns otherwise.
+    ``salts[b]`` (default 0) re-draws sequence b alone: it is generated from
+    ``seed + salts[b] * SALT_STRIDE``."""
+    salts = list(salts) if salts is not None else [0] * cfg.batch
+    seqs = [make_sequence(cfg, seed + salts[b] * SALT_STRIDE, b, with_logits, with_attention)
+            for b in range(cfg.batch)]
     cat = lambda key: np.concatenate([s[key] for s in seqs], axis=0)
     node_off = np.zeros(cfg.batch + 1, dtype=np.int32)
     node_off[1:] = np.cumsum([s["n"] for s in seqs])
     kv_off = np.zeros(cfg.batch + 1, dtype=np.int32)
     kv_off[1:] = np.cumsum([s["kv_len"] for s in seqs])
-    batch = dict(cfg=cfg, seed=seed, node_off=node_off, kv_off=kv_off,
+    batch = dict(cfg=cfg, seed=seed, salts=salts, node_off=node_off, kv_off=kv_off,
                  parent=cat("parent"), token=cat("token"), depth=cat("depth"))
     if with_logits:
         draft, target = cat("draft"), cat("target")

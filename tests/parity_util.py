@@ -12,7 +12,7 @@ GOLD = os.path.join(os.path.dirname(__file__), "golden")
 THRESHOLDS = json.load(open(os.path.join(GOLD, "thresholds.json")))
 
 # guard bands of the float -> integer decisions (the GPU decides in fp32, the oracle in fp64)
-BAND_BIN, BAND_RANK, BAND_PSTAR, BAND_ACCEPT, BAND_CDF = 1e-3, 1e-4, 1e-4, 1e-4, 1e-5
+BAND_BIN, BAND_RANK, BAND_PSTAR, BAND_ACCEPT, BAND_CDF = 1e-3, 1e-4, 1e-4, 1e-4, 5e-7
 
 
 def policy_for(cfg, base=None):
@@ -20,42 +20,51 @@ def policy_for(cfg, base=None):
     return synth.default_policy(cfg, THRESHOLDS[name]["thresholds"])
 
 
+def _sequence_ok(batch, policy, b):
+    """Oracle results of sequence b, or None if one of its float decisions is inside a guard band."""
+    stats, sc = ostep.quantify(batch, policy, b)
+    m = otree.margins(sc, policy)
+    if m["bin"] <= BAND_BIN or m["rank"] <= BAND_RANK or m["pstar"] <= BAND_PSTAR:
+        return None
+    pr = ostep.stratify_prune(batch, policy, b, sc)
+    trace = []
+    acc = ostep.accept_path(batch, b, pr, trace=trace)
+    for t in trace:
+        if t[0] == "accept" and abs(t[2] - t[3]) <= BAND_ACCEPT:
+            return None
+        if t[0] == "final" and (t[1] - t[2] <= BAND_CDF or t[3] - t[1] <= BAND_CDF):
+            return None
+    return dict(stats=stats, scores=sc, pruned=pr, accept=acc)
+
+
 def oracle_case(cfg, policy, seed, attention="full", attn_pairs=64, max_tries=20):
-    """Generates a batch whose every float decision keeps its guard band (else the next seed is
-    taken) and runs the oracle on it.  attention: "full" | "sampled" | "none"."""
-    for s in range(seed, seed + max_tries):
-        batch = synth.make_batch(cfg, s, with_attention=attention != "none")
-        res, ok = [], True
+    """Generates a batch whose every float decision keeps its guard band (a sequence that does
+    not is re-drawn alone with the next salt) and runs the oracle on it.
+    attention: "full" | "sampled" | "none"."""
+    salts = [0] * cfg.batch
+    res = [None] * cfg.batch
+    for _ in range(max_tries):
+        probe = synth.make_batch(cfg, seed, with_attention=False, salts=salts)
         for b in range(cfg.batch):
-            stats, sc = ostep.quantify(batch, policy, b)
-            m = otree.margins(sc, policy)
-            if m["bin"] <= BAND_BIN or m["rank"] <= BAND_RANK or m["pstar"] <= BAND_PSTAR:
-                ok = False
-                break
-            pr = ostep.stratify_prune(batch, policy, b, sc)
-            trace = []
-            acc = ostep.accept_path(batch, b, pr, trace=trace)
-            for t in trace:
-                if t[0] == "accept" and abs(t[2] - t[3]) <= BAND_ACCEPT:
-                    ok = False
-                if t[0] == "final" and (t[1] - t[2] <= BAND_CDF or t[3] - t[1] <= BAND_CDF):
-                    ok = False
-            if not ok:
-                break
-            res.append(dict(stats=stats, scores=sc, pruned=pr, accept=acc))
-        if not ok:
-            continue
-        if attention != "none":
-            rng = np.random.default_rng(s)
-            for b, r in enumerate(res):
-                nk = len(r["pruned"]["keep_idx"])
-                pairs = None
-                if attention == "sampled":
-                    pairs = [(int(rng.integers(nk)), int(rng.integers(cfg.hq))) for _ in range(attn_pairs)]
-                    pairs += [(nk - 1, h) for h in range(0, cfg.hq, max(1, cfg.hq // 8))]
-                r["attn_out"], r["attn_lse"] = ostep.verify_attention(batch, b, r["pruned"], rows=pairs)
-        return batch, res
-    raise RuntimeError("no guard-banded seed found")
+            if res[b] is None:
+                res[b] = _sequence_ok(probe, policy, b)
+                if res[b] is None:
+                    salts[b] += 1
+        if all(r is not None for r in res):
+            break
+    else:
+        raise RuntimeError("no guard-banded draw found")
+    batch = synth.make_batch(cfg, seed, with_attention=attention != "none", salts=salts)
+    if attention != "none":
+        rng = np.random.default_rng(seed)
+        for b, r in enumerate(res):
+            nk = len(r["pruned"]["keep_idx"])
+            pairs = None
+            if attention == "sampled":
+                pairs = [(int(rng.integers(nk)), int(rng.integers(cfg.hq))) for _ in range(attn_pairs)]
+                pairs += [(nk - 1, h) for h in range(0, cfg.hq, max(1, cfg.hq // 8))]
+            r["attn_out"], r["attn_lse"] = ostep.verify_attention(batch, b, r["pruned"], rows=pairs)
+    return batch, res
 
 
 def rel_close(got, want, rel=1e-4, abs_=1e-6):
