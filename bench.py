@@ -52,7 +52,7 @@ class ClockSampler:
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.Q}",
-                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                       "--format=csv,noheader,nounits", "-lms", "50"],
                                       stdout=self.f, stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
@@ -83,6 +83,27 @@ class ClockSampler:
             out = {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
                    "samples": len(sm)}
         return out
+
+
+def rank_seed(rank):
+    """Seed of the batch a rank verifies: every rank gets its own independent trees."""
+    return int(rank)
+
+
+def max_over_ranks(values, device, world):
+    """Element-wise maximum of a list of floats over all ranks (the slowest rank defines the time)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_value(world, batch_per_rank, steps, ms):
+    """Trees verified per second by all ranks together: units all ranks processed / slowest rank's time."""
+    return world * batch_per_rank * steps / (ms * 1e-3)
 
 
 def oracle_sample(batch, policy, ostep):
@@ -156,7 +177,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     policy = load_policy(cfg, synth)
-    batch = synth.make_batch(cfg, rank)                      # each rank verifies its own trees
+    batch = synth.make_batch(cfg, rank_seed(rank))           # each rank verifies its own trees
     db0 = gstep.upload(batch, dev)
     per_set = db0.nbytes()
     R = args.rotate or max(2, -(-2 * L2_BYTES // per_set) + 1)
@@ -248,10 +269,7 @@ def main():
     e2e_s = time.perf_counter() - t0
     barrier()
 
-    if world > 1:
-        t = torch.tensor([ms, e2e_s], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_s = float(t[0]), float(t[1])
+    ms, e2e_s = max_over_ranks([ms, e2e_s], dev, world)
     dev_err = hb.hs_device_error(ctx)
     if rank != 0:
         if world > 1:
@@ -279,7 +297,7 @@ def main():
         traffic = json.load(open(tpath)).get(cfg.name, {}).get("quantify_kernel")
     achieved = kern["quantify"]["gbs"]
     line = {
-        "metric": METRIC, "value": world * cfg.batch * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": whole_job_value(world, cfg.batch, args.steps, ms), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": cfg.name, "batch_per_gpu": cfg.batch, "tree_nodes": n_rows, "kept_nodes": nk,
