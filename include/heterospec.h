@@ -54,7 +54,8 @@ typedef enum {
     HS_ERR_WORKSPACE = 4,   /* workspace given to hs_create is too small for this call */
     HS_ERR_CUDA = 5,        /* a CUDA runtime or driver call failed */
     HS_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired (device status word) */
-    HS_ERR_BAD_TREE = 7     /* device status word: malformed tree or token out of range */
+    HS_ERR_BAD_TREE = 7,    /* device status word: malformed tree or token out of range */
+    HS_ERR_STATIC_LIMIT = 8 /* hs_entropy_quantify_static: batch larger than the built-in scratch array */
 } hs_status;
 
 typedef enum { HS_F32 = 0, HS_BF16 = 1 } hs_dtype;
@@ -172,6 +173,25 @@ typedef struct {
 hs_status hs_entropy_quantify(hs_ctx* ctx, const hs_tree_batch* tree, const void* draft_logits,
                               hs_dtype dtype, int64_t row_stride, int32_t vocab,
                               const hs_policy* policy, const hs_quant_out* out, hs_stream stream);
+
+/* No counterpart in the paper: hs_entropy_quantify for callers that must not allocate device memory
+ * (a process whose memory is owned by one arena fixed at start-up, a component that is forbidden
+ * cudaMalloc after initialisation).  It needs no hs_ctx and calls no cudaMalloc, cudaFree or other
+ * allocating routine: its scratch (chunk partials and arrival counters) is one array built into the
+ * library, about 580 KB that every GPU loading the library holds until the process exits.  Same
+ * arguments, outputs and results as hs_entropy_quantify, on the CURRENT device.
+ *   Limits: n_nodes_total <= HS_STATIC_MAX_ROWS, batch <= HS_STATIC_MAX_BATCH, vocab <= 262144 (bf16) or
+ *   131072 (f32); anything larger returns HS_ERR_STATIC_LIMIT and launches nothing.
+ *   The first call on a device looks up the array's device address (once per device, with that device
+ *   current); make that first call outside any stream capture.
+ *   All calls share the one array: it keeps the previous call's contents (the counters are cleared on the
+ *   stream before each launch), and two calls whose kernels overlap on the GPU - different streams, or
+ *   different threads - race on it.  Serialise them. */
+#define HS_STATIC_MAX_ROWS 256
+#define HS_STATIC_MAX_BATCH 64
+hs_status hs_entropy_quantify_static(const hs_tree_batch* tree, const void* draft_logits, hs_dtype dtype,
+                                     int64_t row_stride, int32_t vocab, const hs_policy* policy,
+                                     const hs_quant_out* out, hs_stream stream);
 
 /* Sec. 4.2-4.3 and the reranking of Sec. 2.2.  Reads score, phi_star, depth, status of `quant`. */
 hs_status hs_stratify_prune(hs_ctx* ctx, const hs_tree_batch* tree, const hs_quant_out* quant,

@@ -60,7 +60,8 @@ class _AcceptOut(C.Structure):
 
 
 EXPORTS = ("hs_status_string", "hs_workspace_bytes", "hs_create", "hs_destroy", "hs_device_error", "hs_entropy_quantify",
-           "hs_stratify_prune", "hs_tree_verify_attention", "hs_accept_path", "hs_philox_uniforms")
+           "hs_stratify_prune", "hs_tree_verify_attention", "hs_accept_path", "hs_philox_uniforms",
+           "hs_entropy_quantify_static")
 
 
 def lib() -> C.CDLL:
@@ -79,6 +80,8 @@ def lib() -> C.CDLL:
         L.hs_device_error.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
         L.hs_entropy_quantify.argtypes = [C.c_void_p, C.POINTER(_TreeBatch), vp, C.c_int, C.c_int64, C.c_int32,
                                           C.POINTER(_Policy), C.POINTER(_QuantOut), vp]
+        L.hs_entropy_quantify_static.argtypes = [C.POINTER(_TreeBatch), vp, C.c_int, C.c_int64, C.c_int32,
+                                                 C.POINTER(_Policy), C.POINTER(_QuantOut), vp]
         L.hs_stratify_prune.argtypes = [C.c_void_p, C.POINTER(_TreeBatch), C.POINTER(_QuantOut),
                                         C.POINTER(_Policy), C.POINTER(_PrunedTree), vp]
         L.hs_tree_verify_attention.argtypes = [C.c_void_p, C.POINTER(_PrunedTree), C.POINTER(_AttnDesc), vp, vp, vp,
@@ -235,6 +238,23 @@ def hs_entropy_quantify(ctx: Context, tree: TreeBatch, draft_logits: torch.Tenso
     _check(lib().hs_entropy_quantify(ctx.handle, C.byref(t), _ptr(draft_logits), _dtype_code(draft_logits),
                                      draft_logits.stride(0), draft_logits.shape[1], C.byref(p), C.byref(o), _stream()),
            "hs_entropy_quantify")
+    return out
+
+
+HS_STATIC_MAX_ROWS, HS_STATIC_MAX_BATCH, HS_ERR_STATIC_LIMIT = 256, 64, 8
+
+
+def hs_entropy_quantify_static(tree: TreeBatch, draft_logits: torch.Tensor, policy: dict,
+                               out: Optional[QuantOut] = None) -> QuantOut:
+    """hs_entropy_quantify without a context: for callers that may not allocate device memory.  The scratch
+    is an array built into the library (limits HS_STATIC_MAX_ROWS / HS_STATIC_MAX_BATCH); the outputs are
+    still the caller's.  Runs on the current device; calls must not overlap on the GPU."""
+    if out is None:
+        out = QuantOut(tree.n_nodes_total, tree.batch, policy["top_k"], draft_logits.device)
+    t, p, o = tree.c(), make_policy(policy), out.c()
+    _check(lib().hs_entropy_quantify_static(C.byref(t), _ptr(draft_logits), _dtype_code(draft_logits),
+                                            draft_logits.stride(0), draft_logits.shape[1], C.byref(p), C.byref(o),
+                                            _stream()), "hs_entropy_quantify_static")
     return out
 
 

@@ -14,6 +14,7 @@ extern "C" const char* hs_status_string(hs_status s) {
         case HS_ERR_CUDA: return "CUDA error";
         case HS_ERR_TIMEOUT: return "device-side wait expired";
         case HS_ERR_BAD_TREE: return "malformed tree";
+        case HS_ERR_STATIC_LIMIT: return "batch exceeds the built-in scratch of the allocation-free entry point";
     }
     return "unknown status";
 }

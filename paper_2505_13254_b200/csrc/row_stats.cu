@@ -11,6 +11,8 @@
 // meta-path Top-K entropy Phi (Eq. 1) and the operational path P* (Sec. 4.1) of that tree.
 #include <math_constants.h>
 
+#include <mutex>
+
 #include "hs_common.cuh"
 #include "hs_layout.h"
 
@@ -430,6 +432,93 @@ hs_status hs_launch_quantify(hs_ctx* ctx, const hs_tree_batch* tree, const void*
     p.pstar_mode = policy->pstar_mode;
     p.entropy_mode = policy->entropy_mode;
     p.is_bf16 = dtype == HS_BF16;
+    dim3 grid(p.chunks, p.rows);
+    if (dtype == HS_BF16) quantify_kernel<true><<<grid, HS_ROW_THREADS, 0, stream>>>(p);
+    else quantify_kernel<false><<<grid, HS_ROW_THREADS, 0, stream>>>(p);
+    return cudaGetLastError() == cudaSuccess ? HS_OK : HS_ERR_CUDA;
+}
+
+// ---- hs_entropy_quantify_static: the same pass without any allocated workspace -------------------------------
+//
+// Some hosts of this library may not allocate device memory at all: a serving process that hands
+// its whole memory budget to one arena at start-up, or code running under a capture / real-time
+// rule that forbids cudaMalloc.  For them the chunk partials and arrival counters of the pass live
+// in one fixed array that is part of the library image, so every GPU that loads the library carries
+// HS_STATIC_SCRATCH_BYTES of it until the process exits.
+#define HS_STATIC_MAX_CHUNKS 16
+#define HS_STATIC_COUNTER_BYTES 2048    // (HS_STATIC_MAX_ROWS + HS_STATIC_MAX_BATCH) ints, rounded up
+#define HS_STATIC_STATS_BYTES (HS_STATIC_MAX_ROWS * HS_STATIC_MAX_CHUNKS * 16)
+#define HS_STATIC_KEYS_BYTES (HS_STATIC_MAX_ROWS * HS_STATIC_MAX_CHUNKS * HS_MAX_TOPK * 8)
+#define HS_STATIC_SCRATCH_BYTES (HS_STATIC_COUNTER_BYTES + HS_STATIC_STATS_BYTES + HS_STATIC_KEYS_BYTES)
+#define HS_STATIC_MAX_DEVICES 64
+
+static __device__ __align__(256) unsigned char g_static_scratch[HS_STATIC_SCRATCH_BYTES];
+// Device address of g_static_scratch on each device.  In host code the symbol itself is only a
+// handle, never an address a kernel may use: the address is asked for once per device.
+static unsigned char* g_static_addr[HS_STATIC_MAX_DEVICES];
+static std::mutex g_static_mutex;
+
+extern "C" hs_status hs_entropy_quantify_static(const hs_tree_batch* tree, const void* draft_logits, hs_dtype dtype,
+                                                int64_t row_stride, int32_t vocab, const hs_policy* policy,
+                                                const hs_quant_out* out, hs_stream stream_) {
+    cudaStream_t stream = (cudaStream_t)stream_;
+    if (!tree || !policy || !out || !draft_logits || ((uintptr_t)draft_logits & 15)) return HS_ERR_INVALID_ARG;
+    if (dtype != HS_F32 && dtype != HS_BF16) return HS_ERR_INVALID_ARG;
+    if (tree->batch < 1 || tree->n_nodes_total < tree->batch || !tree->node_off || !tree->parent || !tree->token)
+        return HS_ERR_INVALID_ARG;
+    const int ve = hs_vec_elems(dtype);
+    if (vocab < 1 || row_stride < vocab || row_stride % ve != 0) return HS_ERR_INVALID_ARG;
+    if (policy->top_k < 1 || policy->top_k > HS_MAX_TOPK || policy->d_base < 0 || policy->phi_mode < 0 ||
+        policy->phi_mode > 1 || policy->pstar_mode < 0 || policy->pstar_mode > 1 || policy->entropy_mode < 0 ||
+        policy->entropy_mode > 1)
+        return HS_ERR_INVALID_ARG;
+    if (!out->row_max || !out->row_lse || !out->h_full || !out->i_topk || !out->i_trunc || !out->topk_val ||
+        !out->topk_idx || !out->logc || !out->score || !out->phi || !out->depth || !out->pstar_node ||
+        !out->phi_star || !out->status)
+        return HS_ERR_INVALID_ARG;
+    const int chunks = hs_row_chunks(vocab, dtype);
+    if (tree->n_nodes_total > HS_STATIC_MAX_ROWS || tree->batch > HS_STATIC_MAX_BATCH || chunks > HS_STATIC_MAX_CHUNKS)
+        return HS_ERR_STATIC_LIMIT;
+
+    int dev = -1;
+    HS_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= HS_STATIC_MAX_DEVICES) return HS_ERR_UNSUPPORTED;
+    unsigned char* base;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_addr[dev]) {              // first call on this device (it is the current one)
+            void* sym = nullptr;
+            if (cudaGetSymbolAddress(&sym, g_static_scratch) != cudaSuccess || !sym) return HS_ERR_CUDA;
+            g_static_addr[dev] = (unsigned char*)sym;
+        }
+        base = g_static_addr[dev];
+    }
+
+    QuantParams p;
+    p.logits = draft_logits;
+    p.row_stride = row_stride;
+    p.vocab = vocab;
+    p.nvec = (vocab + ve - 1) / ve;
+    p.chunks = chunks;
+    p.chunk_vecs = (p.nvec + p.chunks - 1) / p.chunks;
+    p.rows = tree->n_nodes_total;
+    p.batch = tree->batch;
+    p.node_off = tree->node_off;
+    p.parent = tree->parent;
+    p.token = tree->token;
+    p.out = *out;
+    p.row_cnt = (int*)base;
+    p.tree_cnt = (int*)base + HS_STATIC_MAX_ROWS;
+    p.part_stats = (float4*)(base + HS_STATIC_COUNTER_BYTES);
+    p.part_keys = (unsigned long long*)(base + HS_STATIC_COUNTER_BYTES + HS_STATIC_STATS_BYTES);
+    p.K = policy->top_k;
+    p.d_base = policy->d_base;
+    p.phi_mode = policy->phi_mode;
+    p.pstar_mode = policy->pstar_mode;
+    p.entropy_mode = policy->entropy_mode;
+    p.is_bf16 = dtype == HS_BF16;
+    // The array keeps whatever the previous call left: the arrival counters must start at zero.
+    HS_CUDA_OK(cudaMemsetAsync(base, 0, HS_STATIC_COUNTER_BYTES, stream));
     dim3 grid(p.chunks, p.rows);
     if (dtype == HS_BF16) quantify_kernel<true><<<grid, HS_ROW_THREADS, 0, stream>>>(p);
     else quantify_kernel<false><<<grid, HS_ROW_THREADS, 0, stream>>>(p);
