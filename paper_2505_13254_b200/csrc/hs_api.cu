@@ -1,4 +1,6 @@
 // C-ABI entry points: context, argument validation, dispatch to the kernel launchers.
+#include <stdlib.h>
+
 #include <new>
 
 #include "hs_common.cuh"
@@ -63,6 +65,8 @@ extern "C" hs_status hs_create(hs_ctx** out, int32_t device, size_t workspace_by
         cudaFree(p); delete c; return HS_ERR_CUDA;
     }
     c->encode_tiled = fn;
+    const char* no_pdl = getenv("HS_DISABLE_PDL");
+    c->pdl = !(no_pdl && no_pdl[0] == '1');
     HS_CUDA_OK(cudaDeviceSynchronize());
     *out = c;
     return HS_OK;
