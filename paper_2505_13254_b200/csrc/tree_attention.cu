@@ -405,6 +405,333 @@ tree_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, co
     cluster.sync();      // nobody leaves while its shared memory may still be read
 }
 
+
+// =====================================================================================================
+// tcgen05 version: S = Q K^T and O += P V by the 5th-generation tensor cores, accumulators in tensor
+// memory.  128 threads; thread t owns query row t of the block (= tensor-memory lane t), so the
+// softmax needs no shuffles.  Per 64-key tile: thread 0 has issued S = Q K^T (8 instructions of
+// K = 16, operands straight from the swizzled TMA tiles: Q and K are K-major) and committed to an
+// mbarrier; every thread waits, loads its row of S from tensor memory, masks, exponentiates, writes
+// its row of P (bf16) to a swizzled shared-memory tile; after a barrier thread 0 issues O += P V
+// (V is the MN-major operand, the same swizzled tile as it arrived by TMA) and S of the next tile.
+// O is rescaled in tensor memory only when a row's running maximum grows.
+// =====================================================================================================
+#define UM_THREADS 128
+#define UM_P_BYTES (ATT_BM * ATT_BN * 2)             // 16 KiB: P tile, 128 rows x 64 keys bf16
+#define UM_TMEM_COLS 256                             // S: columns 0..63, O: columns 128..255
+#define UM_SMEM_BYTES (ATT_STAGES * ATT_STAGE_BYTES + ATT_Q_BYTES + UM_P_BYTES + 1024 + 128)
+
+__global__ void __launch_bounds__(UM_THREADS, 1)
+tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV) {
+    extern __shared__ unsigned char smem_raw[];
+    cg::cluster_group cluster = cg::this_cluster();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int pair = blockIdx.z, b = pair / p.hkv, h = pair % p.hkv;
+    const int split = blockIdx.y;
+    const int m0 = blockIdx.x * ATT_BM;
+
+    const unsigned int smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const unsigned int sQ = smem_base + ATT_STAGES * ATT_STAGE_BYTES;
+    const unsigned int sP = sQ + ATT_Q_BYTES;
+    const unsigned int bar0 = sP + UM_P_BYTES;       // full[ATT_STAGES], then S-ready, O-ready, tensor-memory base
+    const unsigned int bar_s = bar0 + ATT_STAGES * 8, bar_o = bar_s + 8, tslot = bar_o + 8;
+    unsigned char* gQ = smem_gen + ATT_STAGES * ATT_STAGE_BYTES;
+    unsigned char* gP = gQ + ATT_Q_BYTES;
+    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + UM_P_BYTES + (ATT_STAGES + 2) * 8);
+
+    // ---- before the dependency wait: barriers, tensor memory, the first KV prefix tiles -----------------
+    const int kv0 = p.kv_off[b];
+    const int L = p.kv_off[b + 1] - kv0;
+    int t_prefix, t0, t1;
+    prefix_range(L, p.nsplit, split, t_prefix, t0, t1);
+    const int np = t1 - t0;
+    auto issue_prefix = [&](int i) {                 // thread 0: tile i of this CTA into stage i % ATT_STAGES
+        const int stage = i % ATT_STAGES;
+        const unsigned int sK = smem_base + stage * ATT_STAGE_BYTES, sV = sK + ATT_TILE_BYTES;
+        const unsigned int bar = bar0 + stage * 8;
+        const int tok = kv0 + (t0 + i) * ATT_BN;
+        mbar_expect_tx(bar, ATT_STAGE_BYTES);
+        if (p.head_first) {
+            tma_load_3d(sK, &tmK, 0, tok, h, bar);
+            tma_load_3d(sK + ATT_TILE_BYTES / 2, &tmK, 64, tok, h, bar);
+            tma_load_3d(sV, &tmV, 0, tok, h, bar);
+            tma_load_3d(sV + ATT_TILE_BYTES / 2, &tmV, 64, tok, h, bar);
+        } else {
+            tma_load_3d(sK, &tmK, 0, h, tok, bar);
+            tma_load_3d(sK + ATT_TILE_BYTES / 2, &tmK, 64, h, tok, bar);
+            tma_load_3d(sV, &tmV, 0, h, tok, bar);
+            tma_load_3d(sV + ATT_TILE_BYTES / 2, &tmV, 64, h, tok, bar);
+        }
+    };
+    const int pre = min(np, ATT_STAGES);
+    if (tid == 0) {
+        for (int i = 0; i < ATT_STAGES + 2; ++i) mbar_init(bar0 + i * 8, 1);
+        mbar_init_fence();
+        for (int i = 0; i < pre; ++i) issue_prefix(i);
+    }
+    if (warp == 0) {
+        tmem_alloc(tslot, UM_TMEM_COLS);
+        tmem_relinquish();
+    }
+    pdl_launch_dependents();
+    pdl_wait();                                      // the pruned tree, q, k_tree, v_tree come from upstream
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const unsigned int tmem_base = *tslot_gen;
+    const unsigned int lane_off = (unsigned int)(warp * 32) << 16;
+    const unsigned int tS = tmem_base, tO = tmem_base + 128;
+
+    const int nk = (p.status[b] == 0) ? p.n_keep[b] : 0;
+    const int M = nk * p.G;
+    if (m0 >= M) {                                   // nothing to do (the same for every CTA of the cluster)
+        if (tid == 0)
+            for (int i = 0; i < pre; ++i) mbar_wait(bar0 + i * 8, 0u, p.err);   // no copy may outlive the CTA
+        __syncthreads();
+        if (warp == 0) tmem_dealloc(tmem_base, UM_TMEM_COLS);
+        return;
+    }
+    const int koff = p.keep_off[b];
+    const int nt_tree = (split == p.nsplit - 1) ? (nk + ATT_BN - 1) / ATT_BN : 0;
+    const int ntiles = np + nt_tree;
+
+    // tree keys/values: gathered rows, 16-byte loads, swizzled stores (2 x 1024 chunks / 128 threads)
+    auto gather_tree = [&](int i) {
+        unsigned char* gK = smem_gen + (i % ATT_STAGES) * ATT_STAGE_BYTES;
+        unsigned char* gV = gK + ATT_TILE_BYTES;
+        const int j0 = (i - np) * ATT_BN;
+#pragma unroll 2
+        for (int it = 0; it < 8; ++it) {
+            const int c = tid + it * UM_THREADS;        // 0..1023
+            const int j = j0 + (c >> 4);
+            uint4 kvv = make_uint4(0, 0, 0, 0), vvv = make_uint4(0, 0, 0, 0);
+            if (j < nk) {
+                const int trow = (p.layout == HS_ROWS_ORIGINAL) ? p.node_off[b] + p.keep_idx[koff + j] : koff + j;
+                const size_t off = ((size_t)trow * p.hkv + h) * HS_HEAD_DIM + (c & 15) * 8;
+                kvv = __ldg(reinterpret_cast<const uint4*>(p.k_tree + off));
+                vvv = __ldg(reinterpret_cast<const uint4*>(p.v_tree + off));
+            }
+            *reinterpret_cast<uint4*>(gK + tile_off(c >> 4, c & 15)) = kvv;
+            *reinterpret_cast<uint4*>(gV + tile_off(c >> 4, c & 15)) = vvv;
+        }
+    };
+
+    // ---- this thread's query row -> shared memory, its ancestor mask and output row ---------------------------
+    const int r = m0 + tid;
+    long long orow = -1;
+    unsigned long long mk0 = 0ull, mk1 = 0ull;
+    {
+        uint4 qv[16];
+#pragma unroll
+        for (int c = 0; c < 16; ++c) qv[c] = make_uint4(0, 0, 0, 0);
+        if (r < M) {
+            const int node = r / p.G, g = r - node * p.G;
+            const int trow = (p.layout == HS_ROWS_ORIGINAL) ? p.node_off[b] + p.keep_idx[koff + node] : koff + node;
+            orow = (long long)trow * p.hq + h * p.G + g;
+            mk0 = p.anc_mask[2 * (size_t)(koff + node)];
+            mk1 = p.anc_mask[2 * (size_t)(koff + node) + 1];
+            const uint4* src = reinterpret_cast<const uint4*>(p.q + (size_t)orow * HS_HEAD_DIM);
+#pragma unroll
+            for (int c = 0; c < 16; ++c) qv[c] = __ldg(src + c);
+        }
+#pragma unroll
+        for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4*>(gQ + q_off(tid, c)) = qv[c];
+    }
+    for (int i = np; i < min(ntiles, ATT_STAGES); ++i) gather_tree(i);     // tree tiles that open the pipeline
+    fence_proxy_async_smem();                        // generic stores -> visible to the tensor cores
+    __syncthreads();
+
+    const unsigned int idesc_qk = umma_idesc_bf16(ATT_BM, ATT_BN, false);
+    const unsigned int idesc_pv = umma_idesc_bf16(ATT_BM, HS_HEAD_DIM, true);
+    // thread 0: S = Q K^T of tile i (waits for the tile if it comes by TMA), then commit to bar_s
+    auto issue_qk = [&](int i) {
+        const int stage = i % ATT_STAGES;
+        if (i < np) mbar_wait(bar0 + stage * 8, (unsigned int)(i / ATT_STAGES) & 1u, p.err);
+        tc_fence_after_sync();
+        const unsigned int sK = smem_base + stage * ATT_STAGE_BYTES;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            const unsigned int koffb = (ks >> 2) * (ATT_TILE_BYTES / 2) + (ks & 3) * 32;
+            const unsigned int qoffb = (ks >> 2) * (ATT_Q_BYTES / 2) + (ks & 3) * 32;
+            umma_ss_bf16(tS, umma_desc_sw128(sQ + qoffb, 16, 1024), umma_desc_sw128(sK + koffb, 16, 1024), idesc_qk,
+                         ks > 0 ? 1u : 0u);
+        }
+        umma_commit(bar_s);
+    };
+    if (tid == 0 && ntiles > 0) issue_qk(0);
+
+    float mrun = -CUDART_INF_F, lrun = 0.f;
+
+    // ---- KV tiles ------------------------------------------------------------------------------------------
+#pragma unroll 1
+    for (int i = 0; i < ntiles; ++i) {
+        mbar_wait(bar_s, (unsigned int)i & 1u, p.err);       // S of tile i is complete, and so is O += P V of tile i - 1
+        tc_fence_after_sync();
+        if (i >= 1) {                                        // the stage of tile i - 1 is free again
+            const int nx = i - 1 + ATT_STAGES;
+            if (nx < ntiles) {
+                if (nx < np) { if (tid == 0) issue_prefix(nx); }
+                else gather_tree(nx);
+            }
+        }
+        unsigned int sr[64];
+        tmem_ld32(tS + lane_off, sr);
+        tmem_ld32(tS + lane_off + 32, sr + 32);
+        tmem_wait_ld();
+
+        const bool is_tree = i >= np;
+        const int col0 = is_tree ? (i - np) * ATT_BN : (t0 + i) * ATT_BN;
+        const int nvis = (is_tree ? nk : L) - col0;          // columns of this tile inside the sequence / tree
+        // a tree tile of 64 keys lies inside one 64-bit word of the ancestor mask
+        unsigned long long vis = nvis >= 64 ? ~0ull : ((1ull << max(nvis, 0)) - 1ull);
+        if (is_tree) vis &= (col0 == 0 ? mk0 : mk1);
+        float mx = -CUDART_INF_F;
+#pragma unroll
+        for (int c = 0; c < 64; ++c) {
+            const float sv = ((vis >> c) & 1ull) ? __uint_as_float(sr[c]) * p.scale_log2 : -CUDART_INF_F;
+            sr[c] = __float_as_uint(sv);
+            mx = fmaxf(mx, sv);
+        }
+        const float mnew = fmaxf(mrun, mx);
+        const float muse = (mnew == -CUDART_INF_F) ? 0.f : mnew;
+        const float corr = ex2_approx(mrun - muse);          // 1 when the maximum did not grow, 0 at the first tile
+        mrun = mnew;
+        // O in tensor memory is rescaled only if some row of this warp needs it (the load/store are warp-wide)
+        if (i > 0 && __any_sync(HS_FULL_MASK, corr != 1.f)) {
+#pragma unroll 1
+            for (int ch = 0; ch < 4; ++ch) {
+                unsigned int ov[32];
+                tmem_ld32(tO + lane_off + ch * 32, ov);
+                tmem_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * corr);
+                tmem_st32(tO + lane_off + ch * 32, ov);
+            }
+            tmem_wait_st();
+        }
+        float lsum = 0.f;
+#pragma unroll
+        for (int c8 = 0; c8 < 8; ++c8) {
+            float pv[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                pv[e] = ex2_approx(__uint_as_float(sr[c8 * 8 + e]) - muse);
+                lsum += pv[e];
+            }
+            uint4 pk;
+            pk.x = pack_bf16(pv[0], pv[1]); pk.y = pack_bf16(pv[2], pv[3]);
+            pk.z = pack_bf16(pv[4], pv[5]); pk.w = pack_bf16(pv[6], pv[7]);
+            *reinterpret_cast<uint4*>(gP + tid * 128 + ((c8 ^ (tid & 7)) << 4)) = pk;
+        }
+        lrun = fmaf(lrun, corr, lsum);
+        fence_proxy_async_smem();                            // P (and gathered tree tiles) -> tensor cores
+        tc_fence_before_sync();
+        __syncthreads();
+        if (tid == 0) {
+            tc_fence_after_sync();
+            const unsigned int sV = smem_base + (i % ATT_STAGES) * ATT_STAGE_BYTES + ATT_TILE_BYTES;
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)                   // 16 keys per instruction: two 8-key groups of V
+                umma_ss_bf16(tO, umma_desc_sw128(sP + kk * 32, 16, 1024),
+                             umma_desc_sw128(sV + kk * 2048, ATT_TILE_BYTES / 2, 1024), idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
+            if (i + 1 < ntiles) issue_qk(i + 1);
+            else umma_commit(bar_o);
+        }
+    }
+    if (ntiles > 0) mbar_wait(bar_o, 0u, p.err);
+    tc_fence_after_sync();
+
+    // ---- epilogue ----------------------------------------------------------------------------------------------
+    if (p.nsplit == 1) {
+        const float inv = lrun > 0.f ? 1.f / lrun : 0.f;
+#pragma unroll 1
+        for (int ch = 0; ch < 4; ++ch) {
+            unsigned int ov[32];
+            tmem_ld32(tO + lane_off + ch * 32, ov);
+            tmem_wait_ld();
+            if (orow >= 0) {
+                uint4* dst = reinterpret_cast<uint4*>(p.out + (size_t)orow * HS_HEAD_DIM + ch * 32);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint4 pk;
+                    pk.x = pack_bf16(__uint_as_float(ov[q * 8 + 0]) * inv, __uint_as_float(ov[q * 8 + 1]) * inv);
+                    pk.y = pack_bf16(__uint_as_float(ov[q * 8 + 2]) * inv, __uint_as_float(ov[q * 8 + 3]) * inv);
+                    pk.z = pack_bf16(__uint_as_float(ov[q * 8 + 4]) * inv, __uint_as_float(ov[q * 8 + 5]) * inv);
+                    pk.w = pack_bf16(__uint_as_float(ov[q * 8 + 6]) * inv, __uint_as_float(ov[q * 8 + 7]) * inv);
+                    dst[q] = pk;
+                }
+            }
+        }
+        if (orow >= 0 && p.lse_out) p.lse_out[orow] = (mrun + log2f(lrun)) * LN2;
+    } else {
+        // ---- merge across the splits of the cluster through distributed shared memory ----------------------------
+        float* po = reinterpret_cast<float*>(smem_gen);                              // [128][ATT_PO_STRIDE]
+        float2* pml = reinterpret_cast<float2*>(smem_gen + ATT_BM * ATT_PO_STRIDE * 4);  // [128] {max (base 2), sum}
+#pragma unroll 1
+        for (int ch = 0; ch < 4; ++ch) {
+            unsigned int ov[32];
+            if (ntiles > 0) { tmem_ld32(tO + lane_off + ch * 32, ov); tmem_wait_ld(); }
+            else {
+#pragma unroll
+                for (int c = 0; c < 32; ++c) ov[c] = 0u;
+            }
+            float4* dst = reinterpret_cast<float4*>(po + tid * ATT_PO_STRIDE + ch * 32);
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                dst[q] = make_float4(__uint_as_float(ov[q * 4]), __uint_as_float(ov[q * 4 + 1]),
+                                     __uint_as_float(ov[q * 4 + 2]), __uint_as_float(ov[q * 4 + 3]));
+        }
+        pml[tid] = make_float2(mrun, lrun);
+        cluster.sync();
+        const int ns = p.nsplit;
+        const int r_lo = split * ATT_BM / ns, r_hi = (split + 1) * ATT_BM / ns;      // rows this CTA merges
+        // items = (row, float4 column); every item reads one float4 from each split
+#pragma unroll 1
+        for (int it = tid; it < (r_hi - r_lo) * 32; it += UM_THREADS) {
+            const int rl = r_lo + (it >> 5), c4 = it & 31;
+            float2 ml[ATT_MAX_SPLIT];
+            float4 v[ATT_MAX_SPLIT];
+#pragma unroll
+            for (int s2 = 0; s2 < ATT_MAX_SPLIT; ++s2) {
+                ml[s2] = make_float2(-CUDART_INF_F, 0.f);
+                v[s2] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (s2 < ns) {
+                    ml[s2] = cluster.map_shared_rank(pml, s2)[rl];
+                    v[s2] = *reinterpret_cast<const float4*>(cluster.map_shared_rank(po, s2) + rl * ATT_PO_STRIDE + c4 * 4);
+                }
+            }
+            float Mx = -CUDART_INF_F;
+#pragma unroll
+            for (int s2 = 0; s2 < ATT_MAX_SPLIT; ++s2) Mx = fmaxf(Mx, ml[s2].x);
+            float lsum = 0.f;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int s2 = 0; s2 < ATT_MAX_SPLIT; ++s2) {
+                const float w = (ml[s2].x == -CUDART_INF_F) ? 0.f : ex2_approx(ml[s2].x - Mx);
+                lsum = fmaf(w, ml[s2].y, lsum);
+                acc.x = fmaf(w, v[s2].x, acc.x); acc.y = fmaf(w, v[s2].y, acc.y);
+                acc.z = fmaf(w, v[s2].z, acc.z); acc.w = fmaf(w, v[s2].w, acc.w);
+            }
+            const int rg = m0 + rl;
+            if (rg < M) {
+                const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+                const int node = rg / p.G, g = rg - node * p.G;
+                const int trow = (p.layout == HS_ROWS_ORIGINAL) ? p.node_off[b] + p.keep_idx[koff + node] : koff + node;
+                const size_t og = (size_t)trow * p.hq + h * p.G + g;
+                uint2 packed;
+                packed.x = pack_bf16(acc.x * inv, acc.y * inv);
+                packed.y = pack_bf16(acc.z * inv, acc.w * inv);
+                *reinterpret_cast<uint2*>(p.out + og * HS_HEAD_DIM + c4 * 4) = packed;
+                if (p.lse_out && c4 == 0) p.lse_out[og] = (Mx + log2f(lsum)) * LN2;
+            }
+        }
+        cluster.sync();      // nobody leaves while its shared memory may still be read
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, UM_TMEM_COLS);
+}
 typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                     const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                     CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -430,15 +757,16 @@ static bool make_kv_map(hs_ctx* ctx, CUtensorMap* tm, const void* base, const hs
     return r == CUDA_SUCCESS;
 }
 
-// KV splits (= cluster size) in {1, 2, 4, 8}: the one with the fewest tile steps on the critical path,
-// waves of CTAs (as many clusters of that size as the device runs at once) times tiles per CTA.
-static int choose_splits(int base_ctas, int sm_count, int prefix_tiles, const int* cluster_cap) {
+// KV splits (= cluster size): the one with the fewest tile steps on the critical path, waves of CTAs (as
+// many clusters of that size as the device runs at once) times tiles per CTA.  `step` = 1 tries 1..8,
+// `step` = 2 only powers of two.
+static int choose_splits(int base_ctas, int sm_count, int prefix_tiles, const int* cluster_cap, bool pow2) {
     int best = 1;
     long best_cost = 0;
-    for (int s = 1, k = 0; s <= ATT_MAX_SPLIT; s *= 2, ++k) {
+    for (int s = 1; s <= ATT_MAX_SPLIT; s = pow2 ? s * 2 : s + 1) {
         if (s > 1 && s > prefix_tiles) break;
         const long ctas = (long)base_ctas * s;
-        const long cap = cluster_cap[k] > 0 ? cluster_cap[k] : sm_count;
+        const long cap = cluster_cap[s] > 0 ? cluster_cap[s] : sm_count;
         const long waves = (ctas + cap - 1) / cap;
         const long cost = waves * ((prefix_tiles + s - 1) / s + 2 + (s > 1 ? 2 : 0));   // + tree tiles, + merge
         if (s == 1 || cost < best_cost) { best_cost = cost; best = s; }
@@ -446,31 +774,40 @@ static int choose_splits(int base_ctas, int sm_count, int prefix_tiles, const in
     return best;
 }
 
+template <typename Kernel>
+static void query_cluster_caps(Kernel kernel, int threads, size_t smem, int sm_count, int* cap) {
+    for (int sz = 1; sz <= ATT_MAX_SPLIT; ++sz) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(1, sz, sm_count);
+        cfg.blockDim = dim3(threads);
+        cfg.dynamicSmemBytes = smem;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = sz; at[0].val.clusterDim.z = 1;
+        cfg.attrs = at;
+        cfg.numAttrs = 1;
+        int nclusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&nclusters, kernel, &cfg) == cudaSuccess) cap[sz] = nclusters * sz;
+        else { cap[sz] = 0; (void)cudaGetLastError(); }
+    }
+}
+
 hs_status hs_launch_attention(hs_ctx* ctx, const hs_pruned_tree* pruned, const hs_attn_desc* d, const void* q,
                               const void* k_tree, const void* v_tree, const void* k_cache, const void* v_cache,
                               void* out, float* lse_out, cudaStream_t stream) {
     static bool attr_set = false;
-    static int cluster_cap[4] = {0, 0, 0, 0};      // CTAs that run at once in clusters of 1, 2, 4, 8
+    static bool legacy = false;                    // HS_ATTN_MMA_SYNC=1: the mma.sync kernel instead of tcgen05
+    static int cap_umma[ATT_MAX_SPLIT + 1], cap_legacy[ATT_MAX_SPLIT + 1];   // CTAs that run at once in clusters of s
     if (!attr_set) {
+        const char* e = getenv("HS_ATTN_MMA_SYNC");
+        legacy = e && e[0] == '1';
         if (cudaFuncSetAttribute(tree_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES) !=
-            cudaSuccess)
+                cudaSuccess ||
+            cudaFuncSetAttribute(tree_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, UM_SMEM_BYTES) !=
+                cudaSuccess)
             return HS_ERR_CUDA;
-        for (int k = 0, sz = 1; k < 4; ++k, sz *= 2) {
-            cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(1, sz, ctx->sm_count);
-            cfg.blockDim = dim3(ATT_THREADS);
-            cfg.dynamicSmemBytes = ATT_SMEM_BYTES;
-            cudaLaunchAttribute at[1];
-            at[0].id = cudaLaunchAttributeClusterDimension;
-            at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = sz; at[0].val.clusterDim.z = 1;
-            cfg.attrs = at;
-            cfg.numAttrs = 1;
-            int nclusters = 0;
-            if (cudaOccupancyMaxActiveClusters(&nclusters, tree_attn_kernel, &cfg) == cudaSuccess)
-                cluster_cap[k] = nclusters * sz;
-            else
-                (void)cudaGetLastError();
-        }
+        query_cluster_caps(tree_attn_kernel, ATT_THREADS, ATT_SMEM_BYTES, ctx->sm_count, cap_legacy);
+        query_cluster_caps(tree_attn_umma_kernel, UM_THREADS, UM_SMEM_BYTES, ctx->sm_count, cap_umma);
         attr_set = true;
     }
     AttnParams p;
@@ -496,7 +833,9 @@ hs_status hs_launch_attention(hs_ctx* ctx, const hs_pruned_tree* pruned, const h
     p.err = ctx->counters + HS_CNT_ERROR;
     const int pairs = d->batch * d->hkv;
     const int mblocks = (p.G * d->max_nodes + ATT_BM - 1) / ATT_BM;
-    p.nsplit = choose_splits(pairs * mblocks, ctx->sm_count, (d->max_kv_len + ATT_BN - 1) / ATT_BN, cluster_cap);
+    const int prefix_tiles = (d->max_kv_len + ATT_BN - 1) / ATT_BN;
+    p.nsplit = legacy ? choose_splits(pairs * mblocks, ctx->sm_count, prefix_tiles, cap_legacy, true)
+                      : choose_splits(pairs * mblocks, ctx->sm_count, prefix_tiles, cap_umma, false);
 
     CUtensorMap tmK, tmV;
     memset(&tmK, 0, sizeof(tmK));
@@ -505,7 +844,9 @@ hs_status hs_launch_attention(hs_ctx* ctx, const hs_pruned_tree* pruned, const h
         if (!make_kv_map(ctx, &tmK, k_cache, d, p.head_first) || !make_kv_map(ctx, &tmV, v_cache, d, p.head_first))
             return HS_ERR_CUDA;
     }
-    cudaError_t e = hs_launch(tree_attn_kernel, dim3(mblocks, p.nsplit, pairs), dim3(ATT_THREADS), ATT_SMEM_BYTES,
-                              stream, ctx->pdl, dim3(1, p.nsplit, 1), p, tmK, tmV);
+    const dim3 grid(mblocks, p.nsplit, pairs), cl(1, p.nsplit, 1);
+    cudaError_t e = legacy
+        ? hs_launch(tree_attn_kernel, grid, dim3(ATT_THREADS), ATT_SMEM_BYTES, stream, ctx->pdl, cl, p, tmK, tmV)
+        : hs_launch(tree_attn_umma_kernel, grid, dim3(UM_THREADS), UM_SMEM_BYTES, stream, ctx->pdl, cl, p, tmK, tmV);
     return e == cudaSuccess ? HS_OK : HS_ERR_CUDA;
 }
