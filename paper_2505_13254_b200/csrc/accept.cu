@@ -18,6 +18,7 @@
 
 #include "hs_common.cuh"
 #include "hs_layout.h"
+#include "hs_ptx.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -76,6 +77,8 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 2) accept_rows_kernel(const Ac
     __shared__ int s_flag;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int chunk = blockIdx.x, k = blockIdx.y, which = blockIdx.z;   // which: 0 target, 1 draft
+    pdl_launch_dependents();
+    pdl_wait();                            // the pruned tree and the logits come from upstream
     if (k >= p.pr.keep_off[p.batch]) return;
     int lo = 0, hi = p.batch;                     // sequence of kept node k
     while (hi - lo > 1) {
@@ -307,6 +310,8 @@ accept_walk_kernel(const AcceptParams p) {
     const int tid = threadIdx.x;
     const int b = blockIdx.x / WALK_CLUSTER;
     const unsigned int rank = cluster.block_rank();
+    pdl_launch_dependents();
+    pdl_wait();                            // arg-max and normalisers come from the row pass
     const int koff = p.pr.keep_off[b];
     const int nk = p.pr.n_keep[b];
     const int nbase = p.node_off[b];
@@ -463,9 +468,12 @@ hs_status hs_launch_accept(hs_ctx* ctx, const hs_tree_batch* tree, const hs_prun
     if (o > ctx->scratch_bytes) return HS_ERR_WORKSPACE;
     p.row_cnt = ctx->counters + HS_CNT_ACC_ROW;
     dim3 grid(p.chunks, rows, 2);
-    if (dtype == HS_BF16) accept_rows_kernel<true><<<grid, HS_ROW_THREADS, 0, stream>>>(p);
-    else accept_rows_kernel<false><<<grid, HS_ROW_THREADS, 0, stream>>>(p);
-    if (cudaGetLastError() != cudaSuccess) return HS_ERR_CUDA;
-    accept_walk_kernel<<<p.batch * WALK_CLUSTER, WALK_THREADS, 0, stream>>>(p);
-    return cudaGetLastError() == cudaSuccess ? HS_OK : HS_ERR_CUDA;
+    cudaError_t e = dtype == HS_BF16
+        ? hs_launch(accept_rows_kernel<true>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p)
+        : hs_launch(accept_rows_kernel<false>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p);
+    if (e != cudaSuccess) return HS_ERR_CUDA;
+    // the cluster shape of the walk is fixed at compile time (__cluster_dims__)
+    e = hs_launch(accept_walk_kernel, dim3(p.batch * WALK_CLUSTER), dim3(WALK_THREADS), 0, stream, ctx->pdl,
+                  dim3(1, 1, 1), p);
+    return e == cudaSuccess ? HS_OK : HS_ERR_CUDA;
 }

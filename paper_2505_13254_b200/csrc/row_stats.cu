@@ -15,6 +15,7 @@
 
 #include "hs_common.cuh"
 #include "hs_layout.h"
+#include "hs_ptx.cuh"
 
 #define CAND_CAP 512
 #define LOG2E 1.4426950408889634f
@@ -138,6 +139,8 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 2) quantify_kernel(const Quant
             d[j] = make_uint4(ninf, ninf, ninf, ninf);
         }
     }
+    pdl_launch_dependents();
+    pdl_wait();            // the loads above are in flight; partials and outputs may still be in use upstream
     // ---- maxima ---------------------------------------------------------------------------
     float vmax[VPT];
     float tmax = -CUDART_INF_F;
@@ -433,9 +436,10 @@ hs_status hs_launch_quantify(hs_ctx* ctx, const hs_tree_batch* tree, const void*
     p.entropy_mode = policy->entropy_mode;
     p.is_bf16 = dtype == HS_BF16;
     dim3 grid(p.chunks, p.rows);
-    if (dtype == HS_BF16) quantify_kernel<true><<<grid, HS_ROW_THREADS, 0, stream>>>(p);
-    else quantify_kernel<false><<<grid, HS_ROW_THREADS, 0, stream>>>(p);
-    return cudaGetLastError() == cudaSuccess ? HS_OK : HS_ERR_CUDA;
+    cudaError_t e = dtype == HS_BF16
+        ? hs_launch(quantify_kernel<true>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p)
+        : hs_launch(quantify_kernel<false>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p);
+    return e == cudaSuccess ? HS_OK : HS_ERR_CUDA;
 }
 
 // ---- hs_entropy_quantify_static: the same pass without any allocated workspace -------------------------------

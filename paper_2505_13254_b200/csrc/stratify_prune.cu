@@ -7,6 +7,7 @@
 // recomputes those counts itself, so no CTA waits for another.
 #include "hs_common.cuh"
 #include "hs_layout.h"
+#include "hs_ptx.cuh"
 
 struct PruneParams {
     int batch;
@@ -54,6 +55,8 @@ __global__ void __launch_bounds__(HS_MAX_NODES) stratify_prune_kernel(const Prun
     __shared__ int s_off;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();                            // scores and Phi(P*) come from the kernel ahead in the stream
     const int base = p.node_off[b];
     const int n = min(p.node_off[b + 1] - base, HS_MAX_NODES);
 
@@ -133,7 +136,6 @@ __global__ void __launch_bounds__(HS_MAX_NODES) stratify_prune_kernel(const Prun
 
 hs_status hs_launch_stratify_prune(hs_ctx* ctx, const hs_tree_batch* tree, const hs_quant_out* quant,
                                    const hs_policy* policy, const hs_pruned_tree* out, cudaStream_t stream) {
-    (void)ctx;
     PruneParams p;
     p.batch = tree->batch;
     p.node_off = tree->node_off;
@@ -148,6 +150,6 @@ hs_status hs_launch_stratify_prune(hs_ctx* ctx, const hs_tree_batch* tree, const
     p.alpha = policy->alpha;
     p.n_default = policy->n_default;
     for (int i = 0; i < 3; ++i) p.gamma_pct[i] = policy->gamma_pct[i];
-    stratify_prune_kernel<<<p.batch, HS_MAX_NODES, 0, stream>>>(p);
-    return cudaGetLastError() == cudaSuccess ? HS_OK : HS_ERR_CUDA;
+    return hs_launch(stratify_prune_kernel, dim3(p.batch), dim3(HS_MAX_NODES), 0, stream, ctx->pdl, dim3(1, 1, 1), p) ==
+                   cudaSuccess ? HS_OK : HS_ERR_CUDA;
 }

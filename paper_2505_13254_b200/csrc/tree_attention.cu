@@ -419,7 +419,9 @@ tree_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, co
 #define UM_THREADS 128
 #define UM_P_BYTES (ATT_BM * ATT_BN * 2)             // 16 KiB: P tile, 128 rows x 64 keys bf16
 #define UM_TMEM_COLS 256                             // S: columns 0..63, O: columns 128..255
-#define UM_SMEM_BYTES (ATT_STAGES * ATT_STAGE_BYTES + ATT_Q_BYTES + UM_P_BYTES + 1024 + 128)
+#define UM_STAGES 3
+#define UM_RECV_BYTES (76 * 1024)                    // partials pushed by the other splits of the cluster
+#define UM_SMEM_BYTES (UM_STAGES * ATT_STAGE_BYTES + ATT_Q_BYTES + UM_P_BYTES + 1024 + UM_RECV_BYTES + 1024)
 
 __global__ void __launch_bounds__(UM_THREADS, 1)
 tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV) {
@@ -432,13 +434,13 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
 
     const unsigned int smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    const unsigned int sQ = smem_base + ATT_STAGES * ATT_STAGE_BYTES;
+    const unsigned int sQ = smem_base + UM_STAGES * ATT_STAGE_BYTES;
     const unsigned int sP = sQ + ATT_Q_BYTES;
-    const unsigned int bar0 = sP + UM_P_BYTES;       // full[ATT_STAGES], then S-ready, O-ready, tensor-memory base
-    const unsigned int bar_s = bar0 + ATT_STAGES * 8, bar_o = bar_s + 8, tslot = bar_o + 8;
-    unsigned char* gQ = smem_gen + ATT_STAGES * ATT_STAGE_BYTES;
+    const unsigned int bar0 = sP + UM_P_BYTES;       // full[UM_STAGES], then S-ready, O-ready, tensor-memory base
+    const unsigned int bar_s = bar0 + UM_STAGES * 8, bar_o = bar_s + 8, tslot = bar_o + 8;
+    unsigned char* gQ = smem_gen + UM_STAGES * ATT_STAGE_BYTES;
     unsigned char* gP = gQ + ATT_Q_BYTES;
-    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + UM_P_BYTES + (ATT_STAGES + 2) * 8);
+    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + UM_P_BYTES + (UM_STAGES + 2) * 8);
 
     // ---- before the dependency wait: barriers, tensor memory, the first KV prefix tiles -----------------
     const int kv0 = p.kv_off[b];
@@ -446,8 +448,8 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     int t_prefix, t0, t1;
     prefix_range(L, p.nsplit, split, t_prefix, t0, t1);
     const int np = t1 - t0;
-    auto issue_prefix = [&](int i) {                 // thread 0: tile i of this CTA into stage i % ATT_STAGES
-        const int stage = i % ATT_STAGES;
+    auto issue_prefix = [&](int i) {                 // thread 0: tile i of this CTA into stage i % UM_STAGES
+        const int stage = i % UM_STAGES;
         const unsigned int sK = smem_base + stage * ATT_STAGE_BYTES, sV = sK + ATT_TILE_BYTES;
         const unsigned int bar = bar0 + stage * 8;
         const int tok = kv0 + (t0 + i) * ATT_BN;
@@ -464,9 +466,9 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
             tma_load_3d(sV + ATT_TILE_BYTES / 2, &tmV, 64, h, tok, bar);
         }
     };
-    const int pre = min(np, ATT_STAGES);
+    const int pre = min(np, UM_STAGES);
     if (tid == 0) {
-        for (int i = 0; i < ATT_STAGES + 2; ++i) mbar_init(bar0 + i * 8, 1);
+        for (int i = 0; i < UM_STAGES + 2; ++i) mbar_init(bar0 + i * 8, 1);
         mbar_init_fence();
         for (int i = 0; i < pre; ++i) issue_prefix(i);
     }
@@ -496,24 +498,35 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     const int nt_tree = (split == p.nsplit - 1) ? (nk + ATT_BN - 1) / ATT_BN : 0;
     const int ntiles = np + nt_tree;
 
-    // tree keys/values: gathered rows, 16-byte loads, swizzled stores (2 x 1024 chunks / 128 threads)
+    // tree keys/values: gathered rows, 16-byte loads (all of a thread's loads in flight together), swizzled
+    // stores; 2 x 1024 chunks / 128 threads
     auto gather_tree = [&](int i) {
-        unsigned char* gK = smem_gen + (i % ATT_STAGES) * ATT_STAGE_BYTES;
+        unsigned char* gK = smem_gen + (i % UM_STAGES) * ATT_STAGE_BYTES;
         unsigned char* gV = gK + ATT_TILE_BYTES;
         const int j0 = (i - np) * ATT_BN;
-#pragma unroll 2
+        uint4 kvv[8], vvv[8];
+        int trow[8];
+#pragma unroll
         for (int it = 0; it < 8; ++it) {
-            const int c = tid + it * UM_THREADS;        // 0..1023
-            const int j = j0 + (c >> 4);
-            uint4 kvv = make_uint4(0, 0, 0, 0), vvv = make_uint4(0, 0, 0, 0);
-            if (j < nk) {
-                const int trow = (p.layout == HS_ROWS_ORIGINAL) ? p.node_off[b] + p.keep_idx[koff + j] : koff + j;
-                const size_t off = ((size_t)trow * p.hkv + h) * HS_HEAD_DIM + (c & 15) * 8;
-                kvv = __ldg(reinterpret_cast<const uint4*>(p.k_tree + off));
-                vvv = __ldg(reinterpret_cast<const uint4*>(p.v_tree + off));
+            const int j = j0 + ((tid + it * UM_THREADS) >> 4);
+            trow[it] = -1;
+            if (j < nk) trow[it] = (p.layout == HS_ROWS_ORIGINAL) ? p.node_off[b] + p.keep_idx[koff + j] : koff + j;
+        }
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            kvv[it] = make_uint4(0, 0, 0, 0);
+            vvv[it] = make_uint4(0, 0, 0, 0);
+            if (trow[it] >= 0) {
+                const size_t off = ((size_t)trow[it] * p.hkv + h) * HS_HEAD_DIM + (tid & 15) * 8;
+                kvv[it] = __ldg(reinterpret_cast<const uint4*>(p.k_tree + off));
+                vvv[it] = __ldg(reinterpret_cast<const uint4*>(p.v_tree + off));
             }
-            *reinterpret_cast<uint4*>(gK + tile_off(c >> 4, c & 15)) = kvv;
-            *reinterpret_cast<uint4*>(gV + tile_off(c >> 4, c & 15)) = vvv;
+        }
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int c = tid + it * UM_THREADS;
+            *reinterpret_cast<uint4*>(gK + tile_off(c >> 4, c & 15)) = kvv[it];
+            *reinterpret_cast<uint4*>(gV + tile_off(c >> 4, c & 15)) = vvv[it];
         }
     };
 
@@ -538,7 +551,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
 #pragma unroll
         for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4*>(gQ + q_off(tid, c)) = qv[c];
     }
-    for (int i = np; i < min(ntiles, ATT_STAGES); ++i) gather_tree(i);     // tree tiles that open the pipeline
+    for (int i = np; i < min(ntiles, UM_STAGES); ++i) gather_tree(i);     // tree tiles that open the pipeline
     fence_proxy_async_smem();                        // generic stores -> visible to the tensor cores
     __syncthreads();
 
@@ -546,8 +559,8 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     const unsigned int idesc_pv = umma_idesc_bf16(ATT_BM, HS_HEAD_DIM, true);
     // thread 0: S = Q K^T of tile i (waits for the tile if it comes by TMA), then commit to bar_s
     auto issue_qk = [&](int i) {
-        const int stage = i % ATT_STAGES;
-        if (i < np) mbar_wait(bar0 + stage * 8, (unsigned int)(i / ATT_STAGES) & 1u, p.err);
+        const int stage = i % UM_STAGES;
+        if (i < np) mbar_wait(bar0 + stage * 8, (unsigned int)(i / UM_STAGES) & 1u, p.err);
         tc_fence_after_sync();
         const unsigned int sK = smem_base + stage * ATT_STAGE_BYTES;
 #pragma unroll
@@ -569,7 +582,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         mbar_wait(bar_s, (unsigned int)i & 1u, p.err);       // S of tile i is complete, and so is O += P V of tile i - 1
         tc_fence_after_sync();
         if (i >= 1) {                                        // the stage of tile i - 1 is free again
-            const int nx = i - 1 + ATT_STAGES;
+            const int nx = i - 1 + UM_STAGES;
             if (nx < ntiles) {
                 if (nx < np) { if (tid == 0) issue_prefix(nx); }
                 else gather_tree(nx);
@@ -630,7 +643,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         __syncthreads();
         if (tid == 0) {
             tc_fence_after_sync();
-            const unsigned int sV = smem_base + (i % ATT_STAGES) * ATT_STAGE_BYTES + ATT_TILE_BYTES;
+            const unsigned int sV = smem_base + (i % UM_STAGES) * ATT_STAGE_BYTES + ATT_TILE_BYTES;
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)                   // 16 keys per instruction: two 8-key groups of V
                 umma_ss_bf16(tO, umma_desc_sw128(sP + kk * 32, 16, 1024),
@@ -666,30 +679,40 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         if (orow >= 0 && p.lse_out) p.lse_out[orow] = (mrun + log2f(lrun)) * LN2;
     } else {
         // ---- merge across the splits of the cluster through distributed shared memory ----------------------------
-        float* po = reinterpret_cast<float*>(smem_gen);                              // [128][ATT_PO_STRIDE]
-        float2* pml = reinterpret_cast<float2*>(smem_gen + ATT_BM * ATT_PO_STRIDE * 4);  // [128] {max (base 2), sum}
-#pragma unroll 1
-        for (int ch = 0; ch < 4; ++ch) {
-            unsigned int ov[32];
-            if (ntiles > 0) { tmem_ld32(tO + lane_off + ch * 32, ov); tmem_wait_ld(); }
-            else {
-#pragma unroll
-                for (int c = 0; c < 32; ++c) ov[c] = 0u;
-            }
-            float4* dst = reinterpret_cast<float4*>(po + tid * ATT_PO_STRIDE + ch * 32);
-#pragma unroll
-            for (int q = 0; q < 8; ++q)
-                dst[q] = make_float4(__uint_as_float(ov[q * 4]), __uint_as_float(ov[q * 4 + 1]),
-                                     __uint_as_float(ov[q * 4 + 2]), __uint_as_float(ov[q * 4 + 3]));
-        }
-        pml[tid] = make_float2(mrun, lrun);
-        cluster.sync();
+        // Row rl of the block is merged by CTA owner(rl) = rl * ns / 128.  Every CTA PUSHES its partial of a row
+        // into the owner's shared memory (remote stores do not stall the sender), then, after a cluster
+        // barrier, every owner merges its rows from its own shared memory.
         const int ns = p.nsplit;
-        const int r_lo = split * ATT_BM / ns, r_hi = (split + 1) * ATT_BM / ns;      // rows this CTA merges
-        // items = (row, float4 column); every item reads one float4 from each split
+        float* po = reinterpret_cast<float*>(gP + UM_P_BYTES + 1024);                // [ns][rows_max][ATT_PO_STRIDE], never touched by the loop
+        const int rows_max = (ATT_BM + ns - 1) / ns + 1;
+        float2* pml = reinterpret_cast<float2*>(po + (size_t)ns * rows_max * ATT_PO_STRIDE);      // [ns][rows_max]
+        {
+            const int owner = tid * ns / ATT_BM;
+            const int r_lo_o = (owner * ATT_BM + ns - 1) / ns;                        // first row of that owner
+            const int slot_row = split * rows_max + (tid - r_lo_o);
+            float* dst_row = cluster.map_shared_rank(po, owner) + (size_t)slot_row * ATT_PO_STRIDE;
+#pragma unroll 1
+            for (int ch = 0; ch < 4; ++ch) {
+                unsigned int ov[32];
+                if (ntiles > 0) { tmem_ld32(tO + lane_off + ch * 32, ov); tmem_wait_ld(); }
+                else {
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) ov[c] = 0u;
+                }
+                float4* dst = reinterpret_cast<float4*>(dst_row + ch * 32);
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    dst[q] = make_float4(__uint_as_float(ov[q * 4]), __uint_as_float(ov[q * 4 + 1]),
+                                         __uint_as_float(ov[q * 4 + 2]), __uint_as_float(ov[q * 4 + 3]));
+            }
+            cluster.map_shared_rank(pml, owner)[slot_row] = make_float2(mrun, lrun);
+        }
+        cluster.sync();
+        const int r_lo = (split * ATT_BM + ns - 1) / ns, r_hi = ((split + 1) * ATT_BM + ns - 1) / ns;   // rows this CTA owns
+        // items = (row, float4 column); every item combines one float4 of each split, all from local shared memory
 #pragma unroll 1
         for (int it = tid; it < (r_hi - r_lo) * 32; it += UM_THREADS) {
-            const int rl = r_lo + (it >> 5), c4 = it & 31;
+            const int rl = it >> 5, c4 = it & 31;
             float2 ml[ATT_MAX_SPLIT];
             float4 v[ATT_MAX_SPLIT];
 #pragma unroll
@@ -697,8 +720,8 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
                 ml[s2] = make_float2(-CUDART_INF_F, 0.f);
                 v[s2] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (s2 < ns) {
-                    ml[s2] = cluster.map_shared_rank(pml, s2)[rl];
-                    v[s2] = *reinterpret_cast<const float4*>(cluster.map_shared_rank(po, s2) + rl * ATT_PO_STRIDE + c4 * 4);
+                    ml[s2] = pml[s2 * rows_max + rl];
+                    v[s2] = *reinterpret_cast<const float4*>(po + (size_t)(s2 * rows_max + rl) * ATT_PO_STRIDE + c4 * 4);
                 }
             }
             float Mx = -CUDART_INF_F;
@@ -713,7 +736,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
                 acc.x = fmaf(w, v[s2].x, acc.x); acc.y = fmaf(w, v[s2].y, acc.y);
                 acc.z = fmaf(w, v[s2].z, acc.z); acc.w = fmaf(w, v[s2].w, acc.w);
             }
-            const int rg = m0 + rl;
+            const int rg = m0 + r_lo + rl;
             if (rg < M) {
                 const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
                 const int node = rg / p.G, g = rg - node * p.G;
@@ -726,7 +749,6 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
                 if (p.lse_out && c4 == 0) p.lse_out[og] = (Mx + log2f(lsum)) * LN2;
             }
         }
-        cluster.sync();      // nobody leaves while its shared memory may still be read
     }
     tc_fence_before_sync();
     __syncthreads();
