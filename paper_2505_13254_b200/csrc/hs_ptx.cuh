@@ -154,3 +154,21 @@ __device__ __forceinline__ void tmem_st32(unsigned int taddr, const unsigned int
           "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
+
+// ---- thread-block clusters: distributed shared memory -------------------------------------------------
+// shared::cluster address of `local_addr` (a shared::cta address of this CTA's window) in CTA `rank`
+__device__ __forceinline__ unsigned int cluster_map_addr(unsigned int local_addr, unsigned int rank) {
+    unsigned int r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+// Bulk copy from this CTA's shared memory into another CTA's (addresses 16-byte aligned, size a multiple
+// of 16); the transferred bytes are signalled on an mbarrier of the destination CTA.
+__device__ __forceinline__ void bulk_push(unsigned int dst_cluster_addr, unsigned int src_addr, unsigned int bytes,
+                                          unsigned int bar_cluster_addr) {
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_cluster_addr), "r"(src_addr), "r"(bytes), "r"(bar_cluster_addr) : "memory");
+}
+// split cluster barrier (every thread of every CTA of the cluster executes both halves once)
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }

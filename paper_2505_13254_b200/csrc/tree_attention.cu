@@ -436,11 +436,11 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const unsigned int sQ = smem_base + UM_STAGES * ATT_STAGE_BYTES;
     const unsigned int sP = sQ + ATT_Q_BYTES;
-    const unsigned int bar0 = sP + UM_P_BYTES;       // full[UM_STAGES], then S-ready, O-ready, tensor-memory base
-    const unsigned int bar_s = bar0 + UM_STAGES * 8, bar_o = bar_s + 8, tslot = bar_o + 8;
+    const unsigned int bar0 = sP + UM_P_BYTES;       // full[UM_STAGES], then S-ready, O-ready, partials-received, tensor-memory base
+    const unsigned int bar_s = bar0 + UM_STAGES * 8, bar_o = bar_s + 8, bar_r = bar_o + 8, tslot = bar_r + 8;
     unsigned char* gQ = smem_gen + UM_STAGES * ATT_STAGE_BYTES;
     unsigned char* gP = gQ + ATT_Q_BYTES;
-    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + UM_P_BYTES + (UM_STAGES + 2) * 8);
+    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + UM_P_BYTES + (UM_STAGES + 3) * 8);
 
     // ---- before the dependency wait: barriers, tensor memory, the first KV prefix tiles -----------------
     const int kv0 = p.kv_off[b];
@@ -468,7 +468,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     };
     const int pre = min(np, UM_STAGES);
     if (tid == 0) {
-        for (int i = 0; i < UM_STAGES + 2; ++i) mbar_init(bar0 + i * 8, 1);
+        for (int i = 0; i < UM_STAGES + 3; ++i) mbar_init(bar0 + i * 8, 1);
         mbar_init_fence();
         for (int i = 0; i < pre; ++i) issue_prefix(i);
     }
@@ -679,38 +679,56 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         if (orow >= 0 && p.lse_out) p.lse_out[orow] = (mrun + log2f(lrun)) * LN2;
     } else {
         // ---- merge across the splits of the cluster through distributed shared memory ----------------------------
-        // Row rl of the block is merged by CTA owner(rl) = rl * ns / 128.  Every CTA PUSHES its partial of a row
-        // into the owner's shared memory (remote stores do not stall the sender), then, after a cluster
-        // barrier, every owner merges its rows from its own shared memory.
+        // Row rl of the block is merged by CTA owner(rl) = rl * ns / 128.  Every CTA stages its partial
+        // {O row, max, sum} in its own shared memory and one thread PUSHES each owner's rows with a bulk
+        // copy that signals the owner's mbarrier; an owner merges once all ns pieces have landed.
         const int ns = p.nsplit;
-        float* po = reinterpret_cast<float*>(gP + UM_P_BYTES + 1024);                // [ns][rows_max][ATT_PO_STRIDE], never touched by the loop
+        float* stage_po = reinterpret_cast<float*>(smem_gen);                        // [128][ATT_PO_STRIDE]: own partial
+        float* po = reinterpret_cast<float*>(gP + UM_P_BYTES + 1024);                // [ns][rows_max][ATT_PO_STRIDE]: received
+        const unsigned int s_recv = sP + UM_P_BYTES + 1024;
         const int rows_max = (ATT_BM + ns - 1) / ns + 1;
-        float2* pml = reinterpret_cast<float2*>(po + (size_t)ns * rows_max * ATT_PO_STRIDE);      // [ns][rows_max]
-        {
-            const int owner = tid * ns / ATT_BM;
-            const int r_lo_o = (owner * ATT_BM + ns - 1) / ns;                        // first row of that owner
-            const int slot_row = split * rows_max + (tid - r_lo_o);
-            float* dst_row = cluster.map_shared_rank(po, owner) + (size_t)slot_row * ATT_PO_STRIDE;
-#pragma unroll 1
-            for (int ch = 0; ch < 4; ++ch) {
-                unsigned int ov[32];
-                if (ntiles > 0) { tmem_ld32(tO + lane_off + ch * 32, ov); tmem_wait_ld(); }
-                else {
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) ov[c] = 0u;
-                }
-                float4* dst = reinterpret_cast<float4*>(dst_row + ch * 32);
-#pragma unroll
-                for (int q = 0; q < 8; ++q)
-                    dst[q] = make_float4(__uint_as_float(ov[q * 4]), __uint_as_float(ov[q * 4 + 1]),
-                                         __uint_as_float(ov[q * 4 + 2]), __uint_as_float(ov[q * 4 + 3]));
-            }
-            cluster.map_shared_rank(pml, owner)[slot_row] = make_float2(mrun, lrun);
-        }
-        cluster.sync();
         const int r_lo = (split * ATT_BM + ns - 1) / ns, r_hi = ((split + 1) * ATT_BM + ns - 1) / ns;   // rows this CTA owns
-        // items = (row, float4 column); every item combines one float4 of each split, all from local shared memory
+        long long* s_og = reinterpret_cast<long long*>(gQ);                          // output row of each owned row (or -1)
+        if (tid == 0) mbar_expect_tx(bar_r, (unsigned int)(ns * (r_hi - r_lo) * ATT_PO_STRIDE * 4));
+        if (tid < r_hi - r_lo) {
+            const int rg = m0 + r_lo + tid;
+            long long og = -1;
+            if (rg < M) {
+                const int node = rg / p.G, g = rg - node * p.G;
+                const int trow = (p.layout == HS_ROWS_ORIGINAL) ? p.node_off[b] + p.keep_idx[koff + node] : koff + node;
+                og = (long long)trow * p.hq + h * p.G + g;
+            }
+            s_og[tid] = og;
+        }
 #pragma unroll 1
+        for (int ch = 0; ch < 4; ++ch) {
+            unsigned int ov[32];
+            if (ntiles > 0) { tmem_ld32(tO + lane_off + ch * 32, ov); tmem_wait_ld(); }
+            else {
+#pragma unroll
+                for (int c = 0; c < 32; ++c) ov[c] = 0u;
+            }
+            float4* dst = reinterpret_cast<float4*>(stage_po + tid * ATT_PO_STRIDE + ch * 32);
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                dst[q] = make_float4(__uint_as_float(ov[q * 4]), __uint_as_float(ov[q * 4 + 1]),
+                                     __uint_as_float(ov[q * 4 + 2]), __uint_as_float(ov[q * 4 + 3]));
+        }
+        *reinterpret_cast<float2*>(stage_po + tid * ATT_PO_STRIDE + HS_HEAD_DIM) = make_float2(mrun, lrun);
+        fence_proxy_async_smem();                            // staged rows -> visible to the copy engine
+        __syncthreads();
+        if (tid < ns) {                                      // thread o: the rows of owner o
+            const int o = tid;
+            const int o_lo = (o * ATT_BM + ns - 1) / ns, o_hi = ((o + 1) * ATT_BM + ns - 1) / ns;
+            if (o_hi > o_lo)
+                bulk_push(cluster_map_addr(s_recv + (unsigned int)(split * rows_max) * ATT_PO_STRIDE * 4, o),
+                          smem_base + (unsigned int)o_lo * ATT_PO_STRIDE * 4, (unsigned int)(o_hi - o_lo) * ATT_PO_STRIDE * 4,
+                          cluster_map_addr(bar_r, o));
+        }
+        mbar_wait(bar_r, 0u, p.err);                         // all ns pieces of this CTA's rows have landed
+        cluster_arrive();                                    // (a CTA may leave only when every copy has landed everywhere)
+        // items = (row, float4 column); every item combines one float4 of each split, all from local shared memory
+#pragma unroll 2
         for (int it = tid; it < (r_hi - r_lo) * 32; it += UM_THREADS) {
             const int rl = it >> 5, c4 = it & 31;
             float2 ml[ATT_MAX_SPLIT];
@@ -720,8 +738,9 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
                 ml[s2] = make_float2(-CUDART_INF_F, 0.f);
                 v[s2] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (s2 < ns) {
-                    ml[s2] = pml[s2 * rows_max + rl];
-                    v[s2] = *reinterpret_cast<const float4*>(po + (size_t)(s2 * rows_max + rl) * ATT_PO_STRIDE + c4 * 4);
+                    const float* row = po + (size_t)(s2 * rows_max + rl) * ATT_PO_STRIDE;
+                    ml[s2] = *reinterpret_cast<const float2*>(row + HS_HEAD_DIM);
+                    v[s2] = *reinterpret_cast<const float4*>(row + c4 * 4);
                 }
             }
             float Mx = -CUDART_INF_F;
@@ -736,19 +755,17 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
                 acc.x = fmaf(w, v[s2].x, acc.x); acc.y = fmaf(w, v[s2].y, acc.y);
                 acc.z = fmaf(w, v[s2].z, acc.z); acc.w = fmaf(w, v[s2].w, acc.w);
             }
-            const int rg = m0 + r_lo + rl;
-            if (rg < M) {
+            const long long og = s_og[rl];
+            if (og >= 0) {
                 const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
-                const int node = rg / p.G, g = rg - node * p.G;
-                const int trow = (p.layout == HS_ROWS_ORIGINAL) ? p.node_off[b] + p.keep_idx[koff + node] : koff + node;
-                const size_t og = (size_t)trow * p.hq + h * p.G + g;
                 uint2 packed;
                 packed.x = pack_bf16(acc.x * inv, acc.y * inv);
                 packed.y = pack_bf16(acc.z * inv, acc.w * inv);
-                *reinterpret_cast<uint2*>(p.out + og * HS_HEAD_DIM + c4 * 4) = packed;
+                *reinterpret_cast<uint2*>(p.out + (size_t)og * HS_HEAD_DIM + c4 * 4) = packed;
                 if (p.lse_out && c4 == 0) p.lse_out[og] = (Mx + log2f(lsum)) * LN2;
             }
         }
+        cluster_wait();
     }
     tc_fence_before_sync();
     __syncthreads();
