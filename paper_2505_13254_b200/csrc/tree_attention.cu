@@ -416,12 +416,13 @@ tree_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, co
 // (V is the MN-major operand, the same swizzled tile as it arrived by TMA) and S of the next tile.
 // O is rescaled in tensor memory only when a row's running maximum grows.
 // =====================================================================================================
-#define UM_THREADS 128
+#define UM_THREADS 160                               // four softmax warps (one query row per thread) + the issuing warp
+#define UM_ROWS_THREADS 128
 #define UM_P_BYTES (ATT_BM * ATT_BN * 2)             // 16 KiB: P tile, 128 rows x 64 keys bf16
-#define UM_TMEM_COLS 256                             // S: columns 0..63, O: columns 128..255
-#define UM_STAGES 3
-#define UM_RECV_BYTES (76 * 1024)                    // partials pushed by the other splits of the cluster
-#define UM_SMEM_BYTES (UM_STAGES * ATT_STAGE_BYTES + ATT_Q_BYTES + UM_P_BYTES + 1024 + UM_RECV_BYTES + 1024)
+#define UM_TMEM_COLS 256                             // S (two buffers): columns 0..127, O: columns 128..255
+#define UM_STAGES 4
+#define UM_RECV_BYTES (76 * 1024)                    // after the tile loop: partials pushed by the splits of the cluster
+#define UM_SMEM_BYTES (UM_STAGES * ATT_STAGE_BYTES + ATT_Q_BYTES + UM_P_BYTES + 1024 + 1024)
 
 __global__ void __launch_bounds__(UM_THREADS, 1)
 tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV) {
@@ -436,11 +437,12 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const unsigned int sQ = smem_base + UM_STAGES * ATT_STAGE_BYTES;
     const unsigned int sP = sQ + ATT_Q_BYTES;
-    const unsigned int bar0 = sP + UM_P_BYTES;       // full[UM_STAGES], then S-ready, O-ready, partials-received, tensor-memory base
-    const unsigned int bar_s = bar0 + UM_STAGES * 8, bar_o = bar_s + 8, bar_r = bar_o + 8, tslot = bar_r + 8;
+    const unsigned int bar0 = sP + UM_P_BYTES;       // full[UM_STAGES], S-ready[2], PV-done, partials-received, P-written, tensor-memory base
+    const unsigned int bar_s = bar0 + UM_STAGES * 8, bar_pv = bar_s + 16, bar_r = bar_pv + 8, bar_p = bar_r + 8,
+                       tslot = bar_p + 8;
     unsigned char* gQ = smem_gen + UM_STAGES * ATT_STAGE_BYTES;
     unsigned char* gP = gQ + ATT_Q_BYTES;
-    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + UM_P_BYTES + (UM_STAGES + 3) * 8);
+    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + UM_P_BYTES + (UM_STAGES + 5) * 8);
 
     // ---- before the dependency wait: barriers, tensor memory, the first KV prefix tiles -----------------
     const int kv0 = p.kv_off[b];
@@ -468,7 +470,8 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     };
     const int pre = min(np, UM_STAGES);
     if (tid == 0) {
-        for (int i = 0; i < UM_STAGES + 3; ++i) mbar_init(bar0 + i * 8, 1);
+        for (int i = 0; i < UM_STAGES + 4; ++i) mbar_init(bar0 + i * 8, 1);
+        mbar_init(bar_p, UM_ROWS_THREADS);               // P of a tile is written: one arrival per softmax thread
         mbar_init_fence();
         for (int i = 0; i < pre; ++i) issue_prefix(i);
     }
@@ -508,7 +511,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         int trow[8];
 #pragma unroll
         for (int it = 0; it < 8; ++it) {
-            const int j = j0 + ((tid + it * UM_THREADS) >> 4);
+            const int j = j0 + ((tid + it * UM_ROWS_THREADS) >> 4);
             trow[it] = -1;
             if (j < nk) trow[it] = (p.layout == HS_ROWS_ORIGINAL) ? p.node_off[b] + p.keep_idx[koff + j] : koff + j;
         }
@@ -524,7 +527,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         }
 #pragma unroll
         for (int it = 0; it < 8; ++it) {
-            const int c = tid + it * UM_THREADS;
+            const int c = tid + it * UM_ROWS_THREADS;
             *reinterpret_cast<uint4*>(gK + tile_off(c >> 4, c & 15)) = kvv[it];
             *reinterpret_cast<uint4*>(gV + tile_off(c >> 4, c & 15)) = vvv[it];
         }
@@ -538,7 +541,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         uint4 qv[16];
 #pragma unroll
         for (int c = 0; c < 16; ++c) qv[c] = make_uint4(0, 0, 0, 0);
-        if (r < M) {
+        if (r < M && warp < 4) {
             const int node = r / p.G, g = r - node * p.G;
             const int trow = (p.layout == HS_ROWS_ORIGINAL) ? p.node_off[b] + p.keep_idx[koff + node] : koff + node;
             orow = (long long)trow * p.hq + h * p.G + g;
@@ -548,16 +551,19 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
 #pragma unroll
             for (int c = 0; c < 16; ++c) qv[c] = __ldg(src + c);
         }
+        if (warp < 4) {
 #pragma unroll
-        for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4*>(gQ + q_off(tid, c)) = qv[c];
+            for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4*>(gQ + q_off(tid, c)) = qv[c];
+        }
     }
-    for (int i = np; i < min(ntiles, UM_STAGES); ++i) gather_tree(i);     // tree tiles that open the pipeline
+    if (warp < 4)
+        for (int i = np; i < min(ntiles, UM_STAGES); ++i) gather_tree(i);  // tree tiles that open the pipeline
     fence_proxy_async_smem();                        // generic stores -> visible to the tensor cores
     __syncthreads();
 
     const unsigned int idesc_qk = umma_idesc_bf16(ATT_BM, ATT_BN, false);
     const unsigned int idesc_pv = umma_idesc_bf16(ATT_BM, HS_HEAD_DIM, true);
-    // thread 0: S = Q K^T of tile i (waits for the tile if it comes by TMA), then commit to bar_s
+    // thread 0: S = Q K^T of tile i into S buffer i & 1 (waits for the tile if it comes by TMA), then commit
     auto issue_qk = [&](int i) {
         const int stage = i % UM_STAGES;
         if (i < np) mbar_wait(bar0 + stage * 8, (unsigned int)(i / UM_STAGES) & 1u, p.err);
@@ -567,30 +573,42 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         for (int ks = 0; ks < 8; ++ks) {
             const unsigned int koffb = (ks >> 2) * (ATT_TILE_BYTES / 2) + (ks & 3) * 32;
             const unsigned int qoffb = (ks >> 2) * (ATT_Q_BYTES / 2) + (ks & 3) * 32;
-            umma_ss_bf16(tS, umma_desc_sw128(sQ + qoffb, 16, 1024), umma_desc_sw128(sK + koffb, 16, 1024), idesc_qk,
-                         ks > 0 ? 1u : 0u);
+            umma_ss_bf16(tS + (i & 1) * ATT_BN, umma_desc_sw128(sQ + qoffb, 16, 1024), umma_desc_sw128(sK + koffb, 16, 1024),
+                         idesc_qk, ks > 0 ? 1u : 0u);
         }
-        umma_commit(bar_s);
+        umma_commit(bar_s + (i & 1) * 8);
     };
-    if (tid == 0 && ntiles > 0) issue_qk(0);
-
     float mrun = -CUDART_INF_F, lrun = 0.f;
 
     // ---- KV tiles ------------------------------------------------------------------------------------------
+    if (tid == UM_ROWS_THREADS) {
+        // The issuing thread: S two tiles ahead of the softmax, O += P V as soon as a P is written, TMA refills.
+        if (ntiles > 0) issue_qk(0);
+        if (ntiles > 1) issue_qk(1);
 #pragma unroll 1
-    for (int i = 0; i < ntiles; ++i) {
-        mbar_wait(bar_s, (unsigned int)i & 1u, p.err);       // S of tile i is complete, and so is O += P V of tile i - 1
-        tc_fence_after_sync();
-        if (i >= 1) {                                        // the stage of tile i - 1 is free again
-            const int nx = i - 1 + UM_STAGES;
-            if (nx < ntiles) {
-                if (nx < np) { if (tid == 0) issue_prefix(nx); }
-                else gather_tree(nx);
+        for (int i = 0; i < ntiles; ++i) {
+            if (i >= 1 && i - 1 + UM_STAGES < np) {          // the stage of tile i - 1 is free once its P V is done
+                mbar_wait(bar_pv, (unsigned int)(i - 1) & 1u, p.err);
+                issue_prefix(i - 1 + UM_STAGES);
             }
+            mbar_wait(bar_p, (unsigned int)i & 1u, p.err);   // P of tile i is in shared memory, S buffer i & 1 is read
+            tc_fence_after_sync();
+            const unsigned int sV = smem_base + (i % UM_STAGES) * ATT_STAGE_BYTES + ATT_TILE_BYTES;
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)                   // 16 keys per instruction: two 8-key groups of V
+                umma_ss_bf16(tO, umma_desc_sw128(sP + kk * 32, 16, 1024),
+                             umma_desc_sw128(sV + kk * 2048, ATT_TILE_BYTES / 2, 1024), idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
+            umma_commit(bar_pv);
+            if (i + 2 < ntiles) issue_qk(i + 2);
         }
+    }
+#pragma unroll 1
+    for (int i = 0; i < ntiles && warp < 4; ++i) {
+        mbar_wait(bar_s + (i & 1) * 8, (unsigned int)(i >> 1) & 1u, p.err);      // S of tile i is complete
+        tc_fence_after_sync();
         unsigned int sr[64];
-        tmem_ld32(tS + lane_off, sr);
-        tmem_ld32(tS + lane_off + 32, sr + 32);
+        tmem_ld32(tS + (i & 1) * ATT_BN + lane_off, sr);
+        tmem_ld32(tS + (i & 1) * ATT_BN + lane_off + 32, sr + 32);
         tmem_wait_ld();
 
         const bool is_tree = i >= np;
@@ -610,6 +628,13 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         const float muse = (mnew == -CUDART_INF_F) ? 0.f : mnew;
         const float corr = ex2_approx(mrun - muse);          // 1 when the maximum did not grow, 0 at the first tile
         mrun = mnew;
+        // What follows touches O, P and the stage of tile i - 1: O += P V of tile i - 1 must be complete.
+        if (i >= 1) {
+            mbar_wait(bar_pv, (unsigned int)(i - 1) & 1u, p.err);
+            tc_fence_after_sync();
+            const int nx = i - 1 + UM_STAGES;                // its stage is free again: a tree tile is gathered here,
+            if (nx < ntiles && nx >= np) gather_tree(nx);    // a prefix tile is requested by the issuing thread
+        }
         // O in tensor memory is rescaled only if some row of this warp needs it (the load/store are warp-wide)
         if (i > 0 && __any_sync(HS_FULL_MASK, corr != 1.f)) {
 #pragma unroll 1
@@ -640,26 +665,17 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         lrun = fmaf(lrun, corr, lsum);
         fence_proxy_async_smem();                            // P (and gathered tree tiles) -> tensor cores
         tc_fence_before_sync();
-        __syncthreads();
-        if (tid == 0) {
-            tc_fence_after_sync();
-            const unsigned int sV = smem_base + (i % UM_STAGES) * ATT_STAGE_BYTES + ATT_TILE_BYTES;
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk)                   // 16 keys per instruction: two 8-key groups of V
-                umma_ss_bf16(tO, umma_desc_sw128(sP + kk * 32, 16, 1024),
-                             umma_desc_sw128(sV + kk * 2048, ATT_TILE_BYTES / 2, 1024), idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
-            if (i + 1 < ntiles) issue_qk(i + 1);
-            else umma_commit(bar_o);
-        }
+        mbar_arrive(bar_p);
     }
-    if (ntiles > 0) mbar_wait(bar_o, 0u, p.err);
+    if (ntiles > 0 && warp < 4) mbar_wait(bar_pv, (unsigned int)(ntiles - 1) & 1u, p.err);
+    __syncwarp();                                        // the issuing warp reconverges (warp-aligned barriers follow)
     tc_fence_after_sync();
 
     // ---- epilogue ----------------------------------------------------------------------------------------------
     if (p.nsplit == 1) {
         const float inv = lrun > 0.f ? 1.f / lrun : 0.f;
 #pragma unroll 1
-        for (int ch = 0; ch < 4; ++ch) {
+        for (int ch = 0; ch < 4 && warp < 4; ++ch) {
             unsigned int ov[32];
             tmem_ld32(tO + lane_off + ch * 32, ov);
             tmem_wait_ld();
@@ -683,12 +699,14 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         // {O row, max, sum} in its own shared memory and one thread PUSHES each owner's rows with a bulk
         // copy that signals the owner's mbarrier; an owner merges once all ns pieces have landed.
         const int ns = p.nsplit;
-        float* stage_po = reinterpret_cast<float*>(smem_gen);                        // [128][ATT_PO_STRIDE]: own partial
-        float* po = reinterpret_cast<float*>(gP + UM_P_BYTES + 1024);                // [ns][rows_max][ATT_PO_STRIDE]: received
-        const unsigned int s_recv = sP + UM_P_BYTES + 1024;
+        // shared memory after the tile loop: [0, 76 KB) partials received from the cluster (others write here,
+        // so only after every CTA of the cluster has left its loop), then this CTA's own staged partial
+        float* po = reinterpret_cast<float*>(smem_gen);                              // [ns][rows_max][ATT_PO_STRIDE]: received
+        float* stage_po = reinterpret_cast<float*>(smem_gen + UM_RECV_BYTES);        // [128][ATT_PO_STRIDE]: own partial
+        const unsigned int s_recv = smem_base, s_stage = smem_base + UM_RECV_BYTES;
         const int rows_max = (ATT_BM + ns - 1) / ns + 1;
         const int r_lo = (split * ATT_BM + ns - 1) / ns, r_hi = ((split + 1) * ATT_BM + ns - 1) / ns;   // rows this CTA owns
-        long long* s_og = reinterpret_cast<long long*>(gQ);                          // output row of each owned row (or -1)
+        long long* s_og = reinterpret_cast<long long*>(gP);                          // output row of each owned row (or -1)
         if (tid == 0) mbar_expect_tx(bar_r, (unsigned int)(ns * (r_hi - r_lo) * ATT_PO_STRIDE * 4));
         if (tid < r_hi - r_lo) {
             const int rg = m0 + r_lo + tid;
@@ -701,7 +719,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
             s_og[tid] = og;
         }
 #pragma unroll 1
-        for (int ch = 0; ch < 4; ++ch) {
+        for (int ch = 0; ch < 4 && warp < 4; ++ch) {
             unsigned int ov[32];
             if (ntiles > 0) { tmem_ld32(tO + lane_off + ch * 32, ov); tmem_wait_ld(); }
             else {
@@ -714,22 +732,23 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
                 dst[q] = make_float4(__uint_as_float(ov[q * 4]), __uint_as_float(ov[q * 4 + 1]),
                                      __uint_as_float(ov[q * 4 + 2]), __uint_as_float(ov[q * 4 + 3]));
         }
-        *reinterpret_cast<float2*>(stage_po + tid * ATT_PO_STRIDE + HS_HEAD_DIM) = make_float2(mrun, lrun);
+        if (warp < 4) *reinterpret_cast<float2*>(stage_po + tid * ATT_PO_STRIDE + HS_HEAD_DIM) = make_float2(mrun, lrun);
         fence_proxy_async_smem();                            // staged rows -> visible to the copy engine
-        __syncthreads();
+        cluster_arrive();                                    // every CTA of the cluster is done with its tiles:
+        cluster_wait();                                      // its stage buffers may now receive partials
         if (tid < ns) {                                      // thread o: the rows of owner o
             const int o = tid;
             const int o_lo = (o * ATT_BM + ns - 1) / ns, o_hi = ((o + 1) * ATT_BM + ns - 1) / ns;
             if (o_hi > o_lo)
                 bulk_push(cluster_map_addr(s_recv + (unsigned int)(split * rows_max) * ATT_PO_STRIDE * 4, o),
-                          smem_base + (unsigned int)o_lo * ATT_PO_STRIDE * 4, (unsigned int)(o_hi - o_lo) * ATT_PO_STRIDE * 4,
+                          s_stage + (unsigned int)o_lo * ATT_PO_STRIDE * 4, (unsigned int)(o_hi - o_lo) * ATT_PO_STRIDE * 4,
                           cluster_map_addr(bar_r, o));
         }
         mbar_wait(bar_r, 0u, p.err);                         // all ns pieces of this CTA's rows have landed
         cluster_arrive();                                    // (a CTA may leave only when every copy has landed everywhere)
         // items = (row, float4 column); every item combines one float4 of each split, all from local shared memory
 #pragma unroll 2
-        for (int it = tid; it < (r_hi - r_lo) * 32; it += UM_THREADS) {
+        for (int it = tid; it < (r_hi - r_lo) * 32 && tid < UM_ROWS_THREADS; it += UM_ROWS_THREADS) {
             const int rl = it >> 5, c4 = it & 31;
             float2 ml[ATT_MAX_SPLIT];
             float4 v[ATT_MAX_SPLIT];
