@@ -34,6 +34,22 @@ def load_policy(cfg, synth):
     return synth.default_policy(cfg, th[cfg.name]["thresholds"])
 
 
+def ncu_traffic(kernel, workload):
+    """DRAM bytes per launch of `kernel` from the committed ncu capture, or None if there is none or the
+    kernel's source has changed since the counters were taken."""
+    import hashlib
+    path = os.path.join(ROOT, "paper_2505_13254_b200", "ncu_traffic.json")
+    if not os.path.exists(path):
+        return None
+    ent = json.load(open(path)).get(kernel, {}).get(workload)
+    if not ent:
+        return None
+    src = os.path.join(ROOT, "paper_2505_13254_b200", "csrc", ent["source"])
+    if hashlib.sha1(open(src, "rb").read()).hexdigest() != ent["source_sha1"]:
+        return None
+    return ent["dram_bytes_per_launch"]
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -144,7 +160,7 @@ def run_reference(args, cfg, synth):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=4000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2_8b")
@@ -291,10 +307,7 @@ def main():
     for k in kern.values():
         k["gbs"] = k["bytes"] / (k["us"] * 1e-6) / 1e9 if k["us"] > 0 else None
         k["frac_of_%s_hbm" % peak_kind] = k["gbs"] / peak if k["gbs"] else None
-    traffic = None
-    tpath = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tpath):
-        traffic = json.load(open(tpath)).get(cfg.name, {}).get("quantify_kernel")
+    traffic = ncu_traffic("quantify_kernel", cfg.name)
     achieved = kern["quantify"]["gbs"]
     line = {
         "metric": METRIC, "value": whole_job_value(world, cfg.batch, args.steps, ms), "unit": UNIT, "n_gpus": world,
@@ -309,7 +322,7 @@ def main():
         "clocks": clocks,
         "e2e": {"value": world * cfg.batch * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": 1e3 * e2e_s / e2e_steps},
-        "gpu_launches": 6 * args.steps,
+        "gpu_launches": 5 * args.steps,
         "roofline": {"kernel": "quantify_kernel (hs_entropy_quantify, one launch per step)", "bound": "hbm",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": peak_kind + " (burst copy figure)", "traffic": traffic,
@@ -318,12 +331,21 @@ def main():
         "calls": kern,
         "device_error_word": dev_err,
     }
+    a_gbs = kern["attention"]["gbs"]
+    line["roofline_attention"] = {"kernel": "tree_attn_umma_kernel (hs_tree_verify_attention, one launch per step)",
+                                  "bound": "hbm", "achieved": a_gbs, "peak": peak, "unit": "GB/s",
+                                  "frac": a_gbs / peak if a_gbs else None, "peak_kind": peak_kind + " (burst copy figure)",
+                                  "traffic": ncu_traffic("tree_attn_umma_kernel", cfg.name),
+                                  "algorithmic_bytes_per_launch": attn_bytes}
     if not args.no_cpu_baseline:
         from oracle import step as ostep
-        t = oracle_sample(batch, policy, ostep)
-        line["cpu_baseline"] = {"value": cfg.batch / t, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
-                                "sample": "the same batch once through the numpy fp64 oracle: all logits rows, "
-                                          "all kept-node attention pairs of one layer (%.1f s)" % t}
+        nrep = 5
+        t = sum(oracle_sample(synth.make_batch(cfg, rank_seed(rank) + 1000 * i) if i else batch, policy, ostep)
+                for i in range(nrep))
+        line["cpu_baseline"] = {"value": nrep * cfg.batch / t, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+                                "sample": "%d batches of this workload (seeds differ) once each through the numpy fp64 "
+                                          "oracle: all logits rows, all kept-node attention pairs of one layer (%.1f s)"
+                                          % (nrep, t)}
     print(json.dumps(line))
     ctx.close()
     if world > 1:
