@@ -300,8 +300,9 @@ def main():
     accept_bytes = nk * cfg.vocab * esz
     kern = {
         "quantify": {"bytes": quant_bytes, "us": call_us["quantify"], "launches_per_step": 1},
-        "attention": {"bytes": attn_bytes, "us": call_us["attention"], "launches_per_step": 2},
-        "accept_path": {"bytes": accept_bytes, "us": call_us["accept_path"], "launches_per_step": 2},
+        "attention": {"bytes": attn_bytes, "us": call_us["attention"], "launches_per_step": 1},
+        "accept_path": {"bytes": accept_bytes, "us": call_us["accept_path"],
+                        "launches_per_step": 2 if db0.any_sampling else 1},
         "prune": {"bytes": 0, "us": call_us["prune"], "launches_per_step": 1},
     }
     for k in kern.values():
@@ -322,7 +323,7 @@ def main():
         "clocks": clocks,
         "e2e": {"value": world * cfg.batch * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": 1e3 * e2e_s / e2e_steps},
-        "gpu_launches": 5 * args.steps,
+        "gpu_launches": (5 if db0.any_sampling else 4) * args.steps,
         "roofline": {"kernel": "quantify_kernel (hs_entropy_quantify, one launch per step)", "bound": "hbm",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": peak_kind + " (burst copy figure)", "traffic": traffic,

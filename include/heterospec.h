@@ -208,7 +208,8 @@ hs_status hs_tree_verify_attention(hs_ctx* ctx, const hs_pruned_tree* pruned, co
 
 /* Sec. 2.1 (sampling) and Sec. 5 (temperature 0).  target_logits rows follow `target_layout`;
  * draft_logits rows are always indexed by original node id (as given to hs_entropy_quantify) and
- * are read only by sequences in rejection mode.  mode[b]: hs_accept_mode; temperature[b] > 0 for
+ * are read only by sequences in rejection mode; a caller whose sequences are all greedy passes NULL
+ * (a rejection-mode sequence then gets status HS_ERR_INVALID_ARG) and saves a launch.  mode[b]: hs_accept_mode; temperature[b] > 0 for
  * rejection mode, applied to both models.  Uniforms: Philox4x32-10 with key = seed, counter =
  * (offset, b, original node id, stream) with stream 0 = accept test of that node, 1 = final draw
  * (node 0); u = (x0 >> 8) * 2^-24.  If `uniforms` is not NULL it overrides the generator:

@@ -36,7 +36,7 @@ struct AcceptParams {
     const void* target;
     const void* draft;
     int64_t row_stride;
-    int vocab, nvec, chunks, chunk_vecs, is_bf16;
+    int vocab, nvec, chunks, chunk_vecs, is_bf16, have_draft;
     int batch, n_nodes_total, target_layout;
     const int* node_off;
     const int* token;
@@ -49,6 +49,7 @@ struct AcceptParams {
     RowOut ro;
     uint4* partials;      // [2][max_rows][chunks] {key lo, key hi, max, sum}
     int* row_cnt;
+    int* seq_cnt;         // [batch] merged target rows of a sequence (zero between launches)
 };
 
 __device__ __forceinline__ float ex2a(float x) {
@@ -68,6 +69,54 @@ __device__ __forceinline__ void unpack_v(const uint4& v, float* x) {
     }
 }
 
+// Greedy acceptance of sequence b by one whole CTA (Sec. 5, temperature 0): from the root, move to the kept
+// child whose token is the arg-max of the current node's target row until no child matches; the bonus
+// token is the arg-max where the walk stops.  tgt_arg was written by other CTAs: read it past L1.
+__device__ void greedy_walk(const AcceptParams& p, int b) {
+    __shared__ int s_child;
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int koff = p.pr.keep_off[b];
+    const int nk = p.pr.n_keep[b];
+    const int nbase = p.node_off[b];
+    const int cap = p.out.path_cap;
+    for (int j = tid; j < cap; j += nthr) {
+        p.out.path_nodes[b * cap + j] = -1;
+        p.out.path_compact[b * cap + j] = -1;
+        p.out.path_tokens[b * cap + j] = -1;
+    }
+    __syncthreads();
+    // this thread's kept nodes: parent and token stay in registers for the whole walk (nk <= 128 <= nthr)
+    int my_par = -2, my_tok = -1;
+    if (tid < nk) {
+        my_par = p.pr.new_parent[koff + tid];
+        my_tok = p.token[nbase + p.pr.keep_idx[koff + tid]];
+    }
+    int cur = 0, len = 0, bonus = -1;
+    for (int step = 0; step < nk; ++step) {
+        const int g = __ldcg(&p.ro.tgt_arg[koff + cur]);
+        if (tid == 0) s_child = 0x7fffffff;
+        __syncthreads();
+        if (tid > cur && my_par == cur && my_tok == g) atomicMin(&s_child, tid);
+        __syncthreads();
+        const int nxt = s_child;
+        __syncthreads();
+        if (tid == 0 && len < cap) {
+            p.out.path_compact[b * cap + len] = cur;
+            p.out.path_nodes[b * cap + len] = p.pr.keep_idx[koff + cur];
+        }
+        if (nxt == 0x7fffffff) { bonus = g; break; }
+        if (tid == 0 && len < cap) p.out.path_tokens[b * cap + len] = g;
+        cur = nxt;
+        ++len;
+    }
+    if (tid == 0) {
+        p.out.accept_len[b] = len;
+        p.out.bonus_token[b] = bonus;
+        p.out.terminal_rank[b] = p.pr.keep_rank[koff + cur];
+        p.out.status[b] = HS_OK;
+    }
+}
+
 template <bool BF16>
 __global__ void __launch_bounds__(HS_ROW_THREADS, 2) accept_rows_kernel(const AcceptParams p) {
     constexpr int VE = BF16 ? 8 : 4;
@@ -79,6 +128,19 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 2) accept_rows_kernel(const Ac
     const int chunk = blockIdx.x, k = blockIdx.y, which = blockIdx.z;   // which: 0 target, 1 draft
     pdl_launch_dependents();
     pdl_wait();                            // the pruned tree and the logits come from upstream
+    // sequences that kept nothing (flagged upstream) get their empty result from CTA (0, b, 0)
+    if (chunk == 0 && which == 0 && k < p.batch && (p.pr.n_keep[k] <= 0 || p.pr.status[k] != 0)) {
+        const int cap = p.out.path_cap;
+        for (int j = tid; j < cap; j += HS_ROW_THREADS) {
+            p.out.path_nodes[k * cap + j] = -1;
+            p.out.path_compact[k * cap + j] = -1;
+            p.out.path_tokens[k * cap + j] = -1;
+        }
+        if (tid == 0) {
+            p.out.accept_len[k] = 0; p.out.bonus_token[k] = -1; p.out.terminal_rank[k] = -1;
+            p.out.status[k] = p.pr.status[k] != 0 ? p.pr.status[k] : HS_ERR_BAD_TREE;
+        }
+    }
     if (k >= p.pr.keep_off[p.batch]) return;
     int lo = 0, hi = p.batch;                     // sequence of kept node k
     while (hi - lo > 1) {
@@ -167,8 +229,9 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 2) accept_rows_kernel(const Ac
         if (s_flag) *cnt = 0;
     }
     __syncthreads();
-    if (!s_flag || warp != 0) return;
+    if (!s_flag) return;
     __threadfence();
+    if (warp == 0) {
     // last chunk of the row: merge (chunks <= 32, one lane per chunk)
     unsigned long long ck = 0ull;
     float cm = -CUDART_INF_F, cs = 0.f;
@@ -192,6 +255,23 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 2) accept_rows_kernel(const Ac
             p.ro.drf_ms[k] = make_float2(M, S);
         }
     }
+    }
+    // ---- greedy sequences finish here: the last target row of a sequence to be merged walks its tree ------
+    if (sampling && !p.have_draft && which == 0 && i == 0 && tid == 0) {
+        // rejection sampling needs the draft distribution: the caller passed none
+        p.out.accept_len[b] = 0; p.out.bonus_token[b] = -1; p.out.terminal_rank[b] = -1;
+        p.out.status[b] = HS_ERR_INVALID_ARG;
+    }
+    if (which != 0 || sampling) return;
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        s_flag = (atomicAdd(&p.seq_cnt[b], 1) == nk - 1);
+        if (s_flag) p.seq_cnt[b] = 0;
+        __threadfence();
+    }
+    __syncthreads();
+    if (s_flag) greedy_walk(p, b);
 }
 
 // ---- the walk ----------------------------------------------------------------------------------
@@ -319,6 +399,7 @@ accept_walk_kernel(const AcceptParams p) {
     const bool sampling = p.mode[b] == HS_ACCEPT_REJECTION;
     const size_t esz = p.is_bf16 ? 2 : 4;
 
+    if (!sampling && nk > 0 && p.pr.status[b] == 0) return;      // greedy sequences were finished by the row pass
     if (rank == 0) {
         for (int j = tid; j < cap; j += WALK_THREADS) {
             p.out.path_nodes[b * cap + j] = -1;
@@ -335,28 +416,7 @@ accept_walk_kernel(const AcceptParams p) {
     }
     __syncthreads();
     int cur = 0, len = 0, bonus = -1;
-    if (!sampling) {
-        if (rank != 0) return;
-        for (int step = 0; step < nk; ++step) {
-            const int g = p.ro.tgt_arg[koff + cur];
-            if (tid == 0) s_child = 0x7fffffff;
-            __syncthreads();
-            for (int j = cur + 1 + tid; j < nk; j += WALK_THREADS)
-                if (p.pr.new_parent[koff + j] == cur && p.token[nbase + p.pr.keep_idx[koff + j]] == g)
-                    atomicMin(&s_child, j);
-            __syncthreads();
-            const int nxt = s_child;
-            __syncthreads();
-            if (tid == 0 && len < cap) {
-                p.out.path_compact[b * cap + len] = cur;
-                p.out.path_nodes[b * cap + len] = p.pr.keep_idx[koff + cur];
-            }
-            if (nxt == 0x7fffffff) { bonus = g; break; }
-            if (tid == 0 && len < cap) p.out.path_tokens[b * cap + len] = g;
-            cur = nxt;
-            ++len;
-        }
-    } else {
+    {
         const float T = p.temperature[b];
         const float invT = LOG2E / T;
         for (int step = 0; step < nk; ++step) {
@@ -446,6 +506,7 @@ hs_status hs_launch_accept(hs_ctx* ctx, const hs_tree_batch* tree, const hs_prun
     if (p.chunks > 32) return HS_ERR_SHAPE;
     p.chunk_vecs = (p.nvec + p.chunks - 1) / p.chunks;
     p.is_bf16 = dtype == HS_BF16;
+    p.have_draft = draft_logits != nullptr;
     p.batch = tree->batch;
     p.n_nodes_total = tree->n_nodes_total;
     p.target_layout = target_layout;
@@ -467,11 +528,14 @@ hs_status hs_launch_accept(hs_ctx* ctx, const hs_tree_batch* tree, const hs_prun
     o += (size_t)(HS_MAX_ROWS + rows) * p.chunks * sizeof(uint4);
     if (o > ctx->scratch_bytes) return HS_ERR_WORKSPACE;
     p.row_cnt = ctx->counters + HS_CNT_ACC_ROW;
-    dim3 grid(p.chunks, rows, 2);
+    p.seq_cnt = ctx->counters + HS_CNT_ACC_SEQ;
+    // without draft logits every sequence must be greedy: no draft rows to scan and no sampling walk
+    dim3 grid(p.chunks, rows, p.have_draft ? 2 : 1);
     cudaError_t e = dtype == HS_BF16
         ? hs_launch(accept_rows_kernel<true>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p)
         : hs_launch(accept_rows_kernel<false>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p);
     if (e != cudaSuccess) return HS_ERR_CUDA;
+    if (!p.have_draft) return HS_OK;
     // the cluster shape of the walk is fixed at compile time (__cluster_dims__)
     e = hs_launch(accept_walk_kernel, dim3(p.batch * WALK_CLUSTER), dim3(WALK_THREADS), 0, stream, ctx->pdl,
                   dim3(1, 1, 1), p);

@@ -14,6 +14,7 @@
 #define HS_CNT_QUANT_ROW 0        // [HS_MAX_ROWS]  chunks of a draft row that have finished
 #define HS_CNT_QUANT_TREE 16384   // [HS_MAX_BATCH] rows of a tree that have finished
 #define HS_CNT_ACC_ROW 20480      // [2*HS_MAX_ROWS] chunks of a target / draft row
+#define HS_CNT_ACC_SEQ 53248      // [HS_MAX_BATCH] merged target rows of a sequence
 #define HS_CNT_ERROR 61440        // [1] sticky device error word (bounded wait expired)
 
 // Vocabulary pass: a CTA of HS_ROW_THREADS threads keeps HS_ROW_VPT 16-byte vectors per thread in

@@ -42,6 +42,7 @@ class DeviceBatch:
     offset: int
     max_nodes: int
     max_kv_len: int
+    any_sampling: bool = True
 
     def nbytes(self) -> int:
         ts = [self.tree.node_off, self.tree.parent, self.tree.token, self.draft, self.target, self.q, self.k_tree,
@@ -60,7 +61,8 @@ def upload(batch: dict, device="cuda:0") -> DeviceBatch:
                        i32(batch["mode"]),
                        torch.from_numpy(np.asarray(batch["temperature"], dtype=np.float32)).to(device),
                        int(batch["philox_seed"]), int(batch["philox_offset"]),
-                       int(np.diff(node_off).max()), int(np.diff(kv_off).max()))
+                       int(np.diff(node_off).max()), int(np.diff(kv_off).max()),
+                       bool(np.any(np.asarray(batch["mode"]) != 0)))
 
 
 class VerifyStep:
@@ -90,7 +92,8 @@ class VerifyStep:
                                            node_off=db.tree.node_off, out=self.attn_out, lse_out=self.attn_lse)
 
     def accept_path(self, db: DeviceBatch):
-        return hb.hs_accept_path(self.ctx, db.tree, self.pruned, db.target, db.draft, db.mode, db.temperature,
+        draft = db.draft if db.any_sampling else None        # greedy-only batches need no draft rows
+        return hb.hs_accept_path(self.ctx, db.tree, self.pruned, db.target, draft, db.mode, db.temperature,
                                  target_layout=hb.HS_ROWS_ORIGINAL, seed=db.seed, offset=db.offset,
                                  path_cap=self.accept.path_cap, out=self.accept)
 
