@@ -118,7 +118,7 @@ __device__ void greedy_walk(const AcceptParams& p, int b) {
 }
 
 template <bool BF16>
-__global__ void __launch_bounds__(HS_ROW_THREADS, 2) accept_rows_kernel(const AcceptParams p) {
+__global__ void __launch_bounds__(HS_ROW_THREADS, 4) accept_rows_kernel(const AcceptParams p) {
     constexpr int VE = BF16 ? 8 : 4;
     constexpr int VPT = HS_ROW_VPT;
     __shared__ float s_w[8][2];

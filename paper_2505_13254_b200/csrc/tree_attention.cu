@@ -416,13 +416,14 @@ tree_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, co
 // (V is the MN-major operand, the same swizzled tile as it arrived by TMA) and S of the next tile.
 // O is rescaled in tensor memory only when a row's running maximum grows.
 // =====================================================================================================
-#define UM_THREADS 160                               // four softmax warps (one query row per thread) + the issuing warp
+#define UM_THREADS 288                               // eight softmax warps (two threads per query row) + the issuing warp
 #define UM_ROWS_THREADS 128
+#define UM_SM_THREADS 256                            // softmax threads: row = tid & 127, column half = tid >> 7
 #define UM_P_BYTES (ATT_BM * ATT_BN * 2)             // 16 KiB: P tile, 128 rows x 64 keys bf16
 #define UM_TMEM_COLS 256                             // S (two buffers): columns 0..127, O: columns 128..255
 #define UM_STAGES 4
 #define UM_RECV_BYTES (76 * 1024)                    // after the tile loop: partials pushed by the splits of the cluster
-#define UM_SMEM_BYTES (UM_STAGES * ATT_STAGE_BYTES + ATT_Q_BYTES + UM_P_BYTES + 1024 + 1024)
+#define UM_SMEM_BYTES (UM_STAGES * ATT_STAGE_BYTES + ATT_Q_BYTES + UM_P_BYTES + 4096 + 1024)
 
 __global__ void __launch_bounds__(UM_THREADS, 1)
 tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV) {
@@ -443,6 +444,8 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     unsigned char* gQ = smem_gen + UM_STAGES * ATT_STAGE_BYTES;
     unsigned char* gP = gQ + ATT_Q_BYTES;
     volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + UM_P_BYTES + (UM_STAGES + 5) * 8);
+    float* s_xch = reinterpret_cast<float*>(gP + UM_P_BYTES + 1024);      // [2][2][128]: half-row maxima (per S buffer)
+    float* s_lx = s_xch + 4 * ATT_BM;                                    // [2][128]: half-row sums at the end
 
     // ---- before the dependency wait: barriers, tensor memory, the first KV prefix tiles -----------------
     const int kv0 = p.kv_off[b];
@@ -471,7 +474,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     const int pre = min(np, UM_STAGES);
     if (tid == 0) {
         for (int i = 0; i < UM_STAGES + 4; ++i) mbar_init(bar0 + i * 8, 1);
-        mbar_init(bar_p, UM_ROWS_THREADS);               // P of a tile is written: one arrival per softmax thread
+        mbar_init(bar_p, UM_SM_THREADS);                 // P of a tile is written: one arrival per softmax thread
         mbar_init_fence();
         for (int i = 0; i < pre; ++i) issue_prefix(i);
     }
@@ -485,7 +488,8 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     __syncthreads();
     tc_fence_after_sync();
     const unsigned int tmem_base = *tslot_gen;
-    const unsigned int lane_off = (unsigned int)(warp * 32) << 16;
+    const unsigned int lane_off = (unsigned int)((warp & 3) * 32) << 16;   // a warp reaches lanes 32 * (warp % 4) ...
+    const int row = tid & (ATT_BM - 1), half = (tid >> 7) & 1;               // the thread's query row and column half
     const unsigned int tS = tmem_base, tO = tmem_base + 128;
 
     const int nk = (p.status[b] == 0) ? p.n_keep[b] : 0;
@@ -502,21 +506,21 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     const int ntiles = np + nt_tree;
 
     // tree keys/values: gathered rows, 16-byte loads (all of a thread's loads in flight together), swizzled
-    // stores; 2 x 1024 chunks / 128 threads
+    // stores; 2 x 1024 chunks / 256 threads
     auto gather_tree = [&](int i) {
         unsigned char* gK = smem_gen + (i % UM_STAGES) * ATT_STAGE_BYTES;
         unsigned char* gV = gK + ATT_TILE_BYTES;
         const int j0 = (i - np) * ATT_BN;
-        uint4 kvv[8], vvv[8];
-        int trow[8];
+        uint4 kvv[4], vvv[4];
+        int trow[4];
 #pragma unroll
-        for (int it = 0; it < 8; ++it) {
-            const int j = j0 + ((tid + it * UM_ROWS_THREADS) >> 4);
+        for (int it = 0; it < 4; ++it) {
+            const int j = j0 + ((tid + it * UM_SM_THREADS) >> 4);
             trow[it] = -1;
             if (j < nk) trow[it] = (p.layout == HS_ROWS_ORIGINAL) ? p.node_off[b] + p.keep_idx[koff + j] : koff + j;
         }
 #pragma unroll
-        for (int it = 0; it < 8; ++it) {
+        for (int it = 0; it < 4; ++it) {
             kvv[it] = make_uint4(0, 0, 0, 0);
             vvv[it] = make_uint4(0, 0, 0, 0);
             if (trow[it] >= 0) {
@@ -526,37 +530,37 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
             }
         }
 #pragma unroll
-        for (int it = 0; it < 8; ++it) {
-            const int c = tid + it * UM_ROWS_THREADS;
+        for (int it = 0; it < 4; ++it) {
+            const int c = tid + it * UM_SM_THREADS;
             *reinterpret_cast<uint4*>(gK + tile_off(c >> 4, c & 15)) = kvv[it];
             *reinterpret_cast<uint4*>(gV + tile_off(c >> 4, c & 15)) = vvv[it];
         }
     };
 
     // ---- this thread's query row -> shared memory, its ancestor mask and output row ---------------------------
-    const int r = m0 + tid;
+    const int r = m0 + row;
     long long orow = -1;
     unsigned long long mk0 = 0ull, mk1 = 0ull;
     {
-        uint4 qv[16];
+        uint4 qv[8];                                     // this thread's half of the row
 #pragma unroll
-        for (int c = 0; c < 16; ++c) qv[c] = make_uint4(0, 0, 0, 0);
-        if (r < M && warp < 4) {
+        for (int c = 0; c < 8; ++c) qv[c] = make_uint4(0, 0, 0, 0);
+        if (r < M && warp < 8) {
             const int node = r / p.G, g = r - node * p.G;
             const int trow = (p.layout == HS_ROWS_ORIGINAL) ? p.node_off[b] + p.keep_idx[koff + node] : koff + node;
             orow = (long long)trow * p.hq + h * p.G + g;
             mk0 = p.anc_mask[2 * (size_t)(koff + node)];
             mk1 = p.anc_mask[2 * (size_t)(koff + node) + 1];
-            const uint4* src = reinterpret_cast<const uint4*>(p.q + (size_t)orow * HS_HEAD_DIM);
+            const uint4* src = reinterpret_cast<const uint4*>(p.q + (size_t)orow * HS_HEAD_DIM) + half * 8;
 #pragma unroll
-            for (int c = 0; c < 16; ++c) qv[c] = __ldg(src + c);
+            for (int c = 0; c < 8; ++c) qv[c] = __ldg(src + c);
         }
-        if (warp < 4) {
+        if (warp < 8) {
 #pragma unroll
-            for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4*>(gQ + q_off(tid, c)) = qv[c];
+            for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(gQ + q_off(row, half * 8 + c)) = qv[c];
         }
     }
-    if (warp < 4)
+    if (warp < 8)
         for (int i = np; i < min(ntiles, UM_STAGES); ++i) gather_tree(i);  // tree tiles that open the pipeline
     fence_proxy_async_smem();                        // generic stores -> visible to the tensor cores
     __syncthreads();
@@ -581,7 +585,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     float mrun = -CUDART_INF_F, lrun = 0.f;
 
     // ---- KV tiles ------------------------------------------------------------------------------------------
-    if (tid == UM_ROWS_THREADS) {
+    if (tid == UM_SM_THREADS) {
         // The issuing thread: S two tiles ahead of the softmax, O += P V as soon as a P is written, TMA refills.
         if (ntiles > 0) issue_qk(0);
         if (ntiles > 1) issue_qk(1);
@@ -603,27 +607,32 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         }
     }
 #pragma unroll 1
-    for (int i = 0; i < ntiles && warp < 4; ++i) {
+    for (int i = 0; i < ntiles && warp < 8; ++i) {
         mbar_wait(bar_s + (i & 1) * 8, (unsigned int)(i >> 1) & 1u, p.err);      // S of tile i is complete
         tc_fence_after_sync();
-        unsigned int sr[64];
-        tmem_ld32(tS + (i & 1) * ATT_BN + lane_off, sr);
-        tmem_ld32(tS + (i & 1) * ATT_BN + lane_off + 32, sr + 32);
+        unsigned int sr[32];                                 // this thread's 32 of the row's 64 scores
+        tmem_ld32(tS + (i & 1) * ATT_BN + half * 32 + lane_off, sr);
         tmem_wait_ld();
 
         const bool is_tree = i >= np;
         const int col0 = is_tree ? (i - np) * ATT_BN : (t0 + i) * ATT_BN;
         const int nvis = (is_tree ? nk : L) - col0;          // columns of this tile inside the sequence / tree
         // a tree tile of 64 keys lies inside one 64-bit word of the ancestor mask
-        unsigned long long vis = nvis >= 64 ? ~0ull : ((1ull << max(nvis, 0)) - 1ull);
-        if (is_tree) vis &= (col0 == 0 ? mk0 : mk1);
+        unsigned long long vis64 = nvis >= 64 ? ~0ull : ((1ull << max(nvis, 0)) - 1ull);
+        if (is_tree) vis64 &= (col0 == 0 ? mk0 : mk1);
+        const unsigned int vis = (unsigned int)(vis64 >> (half * 32));
         float mx = -CUDART_INF_F;
 #pragma unroll
-        for (int c = 0; c < 64; ++c) {
-            const float sv = ((vis >> c) & 1ull) ? __uint_as_float(sr[c]) * p.scale_log2 : -CUDART_INF_F;
+        for (int c = 0; c < 32; ++c) {
+            const float sv = ((vis >> c) & 1u) ? __uint_as_float(sr[c]) * p.scale_log2 : -CUDART_INF_F;
             sr[c] = __float_as_uint(sv);
             mx = fmaxf(mx, sv);
         }
+        // the row maximum of this tile: exchanged between the two threads of a row (one buffer per S buffer)
+        float* xch = s_xch + (i & 1) * 2 * ATT_BM;
+        xch[half * ATT_BM + row] = mx;
+        asm volatile("bar.sync 1, %0;" ::"n"(UM_SM_THREADS) : "memory");
+        mx = fmaxf(mx, xch[(half ^ 1) * ATT_BM + row]);
         const float mnew = fmaxf(mrun, mx);
         const float muse = (mnew == -CUDART_INF_F) ? 0.f : mnew;
         const float corr = ex2_approx(mrun - muse);          // 1 when the maximum did not grow, 0 at the first tile
@@ -635,22 +644,23 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
             const int nx = i - 1 + UM_STAGES;                // its stage is free again: a tree tile is gathered here,
             if (nx < ntiles && nx >= np) gather_tree(nx);    // a prefix tile is requested by the issuing thread
         }
-        // O in tensor memory is rescaled only if some row of this warp needs it (the load/store are warp-wide)
+        // O in tensor memory is rescaled only if some row of this warp needs it (the load/store are warp-wide);
+        // each of a row's two threads rescales its 64 of the 128 columns
         if (i > 0 && __any_sync(HS_FULL_MASK, corr != 1.f)) {
 #pragma unroll 1
-            for (int ch = 0; ch < 4; ++ch) {
+            for (int ch = 0; ch < 2; ++ch) {
                 unsigned int ov[32];
-                tmem_ld32(tO + lane_off + ch * 32, ov);
+                tmem_ld32(tO + lane_off + half * 64 + ch * 32, ov);
                 tmem_wait_ld();
 #pragma unroll
                 for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * corr);
-                tmem_st32(tO + lane_off + ch * 32, ov);
+                tmem_st32(tO + lane_off + half * 64 + ch * 32, ov);
             }
             tmem_wait_st();
         }
         float lsum = 0.f;
 #pragma unroll
-        for (int c8 = 0; c8 < 8; ++c8) {
+        for (int c8 = 0; c8 < 4; ++c8) {
             float pv[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
@@ -660,27 +670,31 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
             uint4 pk;
             pk.x = pack_bf16(pv[0], pv[1]); pk.y = pack_bf16(pv[2], pv[3]);
             pk.z = pack_bf16(pv[4], pv[5]); pk.w = pack_bf16(pv[6], pv[7]);
-            *reinterpret_cast<uint4*>(gP + tid * 128 + ((c8 ^ (tid & 7)) << 4)) = pk;
+            *reinterpret_cast<uint4*>(gP + row * 128 + (((half * 4 + c8) ^ (row & 7)) << 4)) = pk;
         }
-        lrun = fmaf(lrun, corr, lsum);
+        lrun = fmaf(lrun, corr, lsum);                       // the sum over this thread's half of the columns
         fence_proxy_async_smem();                            // P (and gathered tree tiles) -> tensor cores
         tc_fence_before_sync();
         mbar_arrive(bar_p);
     }
-    if (ntiles > 0 && warp < 4) mbar_wait(bar_pv, (unsigned int)(ntiles - 1) & 1u, p.err);
+    if (ntiles > 0 && warp < 8) mbar_wait(bar_pv, (unsigned int)(ntiles - 1) & 1u, p.err);
     __syncwarp();                                        // the issuing warp reconverges (warp-aligned barriers follow)
     tc_fence_after_sync();
+    // the row sum: both halves together
+    if (warp < 8) s_lx[half * ATT_BM + row] = lrun;
+    __syncthreads();
+    if (warp < 8) lrun += s_lx[(half ^ 1) * ATT_BM + row];
 
     // ---- epilogue ----------------------------------------------------------------------------------------------
     if (p.nsplit == 1) {
         const float inv = lrun > 0.f ? 1.f / lrun : 0.f;
 #pragma unroll 1
-        for (int ch = 0; ch < 4 && warp < 4; ++ch) {
+        for (int ch = 0; ch < 2 && warp < 8; ++ch) {
             unsigned int ov[32];
-            tmem_ld32(tO + lane_off + ch * 32, ov);
+            tmem_ld32(tO + lane_off + half * 64 + ch * 32, ov);
             tmem_wait_ld();
             if (orow >= 0) {
-                uint4* dst = reinterpret_cast<uint4*>(p.out + (size_t)orow * HS_HEAD_DIM + ch * 32);
+                uint4* dst = reinterpret_cast<uint4*>(p.out + (size_t)orow * HS_HEAD_DIM + half * 64 + ch * 32);
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     uint4 pk;
@@ -692,7 +706,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
                 }
             }
         }
-        if (orow >= 0 && p.lse_out) p.lse_out[orow] = (mrun + log2f(lrun)) * LN2;
+        if (orow >= 0 && p.lse_out && half == 0) p.lse_out[orow] = (mrun + log2f(lrun)) * LN2;
     } else {
         // ---- merge across the splits of the cluster through distributed shared memory ----------------------------
         // Row rl of the block is merged by CTA owner(rl) = rl * ns / 128.  Every CTA stages its partial
@@ -719,20 +733,20 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
             s_og[tid] = og;
         }
 #pragma unroll 1
-        for (int ch = 0; ch < 4 && warp < 4; ++ch) {
+        for (int ch = 0; ch < 2 && warp < 8; ++ch) {
             unsigned int ov[32];
-            if (ntiles > 0) { tmem_ld32(tO + lane_off + ch * 32, ov); tmem_wait_ld(); }
+            if (ntiles > 0) { tmem_ld32(tO + lane_off + half * 64 + ch * 32, ov); tmem_wait_ld(); }
             else {
 #pragma unroll
                 for (int c = 0; c < 32; ++c) ov[c] = 0u;
             }
-            float4* dst = reinterpret_cast<float4*>(stage_po + tid * ATT_PO_STRIDE + ch * 32);
+            float4* dst = reinterpret_cast<float4*>(stage_po + row * ATT_PO_STRIDE + half * 64 + ch * 32);
 #pragma unroll
             for (int q = 0; q < 8; ++q)
                 dst[q] = make_float4(__uint_as_float(ov[q * 4]), __uint_as_float(ov[q * 4 + 1]),
                                      __uint_as_float(ov[q * 4 + 2]), __uint_as_float(ov[q * 4 + 3]));
         }
-        if (warp < 4) *reinterpret_cast<float2*>(stage_po + tid * ATT_PO_STRIDE + HS_HEAD_DIM) = make_float2(mrun, lrun);
+        if (warp < 4) *reinterpret_cast<float2*>(stage_po + row * ATT_PO_STRIDE + HS_HEAD_DIM) = make_float2(mrun, lrun);
         fence_proxy_async_smem();                            // staged rows -> visible to the copy engine
         cluster_arrive();                                    // every CTA of the cluster is done with its tiles:
         cluster_wait();                                      // its stage buffers may now receive partials
@@ -748,7 +762,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         cluster_arrive();                                    // (a CTA may leave only when every copy has landed everywhere)
         // items = (row, float4 column); every item combines one float4 of each split, all from local shared memory
 #pragma unroll 2
-        for (int it = tid; it < (r_hi - r_lo) * 32 && tid < UM_ROWS_THREADS; it += UM_ROWS_THREADS) {
+        for (int it = tid; it < (r_hi - r_lo) * 32 && tid < UM_SM_THREADS; it += UM_SM_THREADS) {
             const int rl = it >> 5, c4 = it & 31;
             float2 ml[ATT_MAX_SPLIT];
             float4 v[ATT_MAX_SPLIT];
