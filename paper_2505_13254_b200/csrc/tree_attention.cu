@@ -423,7 +423,7 @@ tree_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, co
 #define UM_TMEM_COLS 256                             // S (two buffers): columns 0..127, O: columns 128..255
 #define UM_STAGES 4
 #define UM_RECV_BYTES (76 * 1024)                    // after the tile loop: partials pushed by the splits of the cluster
-#define UM_SMEM_BYTES (UM_STAGES * ATT_STAGE_BYTES + ATT_Q_BYTES + UM_P_BYTES + 4096 + 1024)
+#define UM_SMEM_BYTES (UM_STAGES * ATT_STAGE_BYTES + ATT_Q_BYTES + 2 * UM_P_BYTES + 4096 + 1024)
 
 __global__ void __launch_bounds__(UM_THREADS, 1)
 tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV) {
@@ -438,13 +438,13 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const unsigned int sQ = smem_base + UM_STAGES * ATT_STAGE_BYTES;
     const unsigned int sP = sQ + ATT_Q_BYTES;
-    const unsigned int bar0 = sP + UM_P_BYTES;       // full[UM_STAGES], S-ready[2], PV-done, partials-received, P-written, tensor-memory base
+    const unsigned int bar0 = sP + 2 * UM_P_BYTES;   // (P is double-buffered) full[UM_STAGES], S-ready[2], PV-done, partials-received, P-written, tensor-memory base
     const unsigned int bar_s = bar0 + UM_STAGES * 8, bar_pv = bar_s + 16, bar_r = bar_pv + 8, bar_p = bar_r + 8,
                        tslot = bar_p + 8;
     unsigned char* gQ = smem_gen + UM_STAGES * ATT_STAGE_BYTES;
     unsigned char* gP = gQ + ATT_Q_BYTES;
-    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + UM_P_BYTES + (UM_STAGES + 5) * 8);
-    float* s_xch = reinterpret_cast<float*>(gP + UM_P_BYTES + 1024);      // [2][2][128]: half-row maxima (per S buffer)
+    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + 2 * UM_P_BYTES + (UM_STAGES + 5) * 8);
+    float* s_xch = reinterpret_cast<float*>(gP + 2 * UM_P_BYTES + 1024);      // [2][2][128]: half-row maxima (per S buffer)
     float* s_lx = s_xch + 4 * ATT_BM;                                    // [2][128]: half-row sums at the end
 
     // ---- before the dependency wait: barriers, tensor memory, the first KV prefix tiles -----------------
@@ -600,7 +600,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
             const unsigned int sV = smem_base + (i % UM_STAGES) * ATT_STAGE_BYTES + ATT_TILE_BYTES;
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)                   // 16 keys per instruction: two 8-key groups of V
-                umma_ss_bf16(tO, umma_desc_sw128(sP + kk * 32, 16, 1024),
+                umma_ss_bf16(tO, umma_desc_sw128(sP + (i & 1) * UM_P_BYTES + kk * 32, 16, 1024),
                              umma_desc_sw128(sV + kk * 2048, ATT_TILE_BYTES / 2, 1024), idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
             umma_commit(bar_pv);
             if (i + 2 < ntiles) issue_qk(i + 2);
@@ -617,17 +617,24 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         const bool is_tree = i >= np;
         const int col0 = is_tree ? (i - np) * ATT_BN : (t0 + i) * ATT_BN;
         const int nvis = (is_tree ? nk : L) - col0;          // columns of this tile inside the sequence / tree
-        // a tree tile of 64 keys lies inside one 64-bit word of the ancestor mask
-        unsigned long long vis64 = nvis >= 64 ? ~0ull : ((1ull << max(nvis, 0)) - 1ull);
-        if (is_tree) vis64 &= (col0 == 0 ? mk0 : mk1);
-        const unsigned int vis = (unsigned int)(vis64 >> (half * 32));
+        // The scores stay unscaled in registers (the scale is positive: it commutes with the maximum and folds into
+        // the exponent's multiply-add). A prefix tile inside the sequence needs no mask at all.
         float mx = -CUDART_INF_F;
+        if (!is_tree && nvis >= ATT_BN) {
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-            const float sv = ((vis >> c) & 1u) ? __uint_as_float(sr[c]) * p.scale_log2 : -CUDART_INF_F;
-            sr[c] = __float_as_uint(sv);
-            mx = fmaxf(mx, sv);
+            for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(sr[c]));
+        } else {
+            // a tree tile of 64 keys lies inside one 64-bit word of the ancestor mask
+            unsigned long long vis64 = nvis >= 64 ? ~0ull : ((1ull << max(nvis, 0)) - 1ull);
+            if (is_tree) vis64 &= (col0 == 0 ? mk0 : mk1);
+            const unsigned int vis = (unsigned int)(vis64 >> (half * 32));
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+                if (!((vis >> c) & 1u)) sr[c] = __float_as_uint(-CUDART_INF_F);
+                mx = fmaxf(mx, __uint_as_float(sr[c]));
+            }
         }
+        mx *= p.scale_log2;
         // the row maximum of this tile: exchanged between the two threads of a row (one buffer per S buffer)
         float* xch = s_xch + (i & 1) * 2 * ATT_BM;
         xch[half * ATT_BM + row] = mx;
@@ -637,16 +644,33 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         const float muse = (mnew == -CUDART_INF_F) ? 0.f : mnew;
         const float corr = ex2_approx(mrun - muse);          // 1 when the maximum did not grow, 0 at the first tile
         mrun = mnew;
-        // What follows touches O, P and the stage of tile i - 1: O += P V of tile i - 1 must be complete.
-        if (i >= 1) {
+        // the row's P of this tile, in registers first: nothing has been waited for so far
+        float lsum = 0.f;
+        uint4 pk[4];
+#pragma unroll
+        for (int c8 = 0; c8 < 4; ++c8) {
+            float pv[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                pv[e] = ex2_approx(fmaf(__uint_as_float(sr[c8 * 8 + e]), p.scale_log2, -muse));
+                lsum += pv[e];
+            }
+            pk[c8].x = pack_bf16(pv[0], pv[1]); pk[c8].y = pack_bf16(pv[2], pv[3]);
+            pk[c8].z = pack_bf16(pv[4], pv[5]); pk[c8].w = pack_bf16(pv[6], pv[7]);
+        }
+        // O and the stage of tile i - 1 may be touched only when O += P V of tile i - 1 is complete; that is
+        // needed when a tree tile is gathered into the stage or when O has to be rescaled (the load/store are
+        // warp-wide: a warp rescales if any of its rows needs it; each of a row's two threads does 64 columns).
+        // P itself is double-buffered: buffer i & 1 was last read by tile i - 2, complete since S of tile i is.
+        const int nx = i - 1 + UM_STAGES;
+        const bool do_gather = i >= 1 && nx < ntiles && nx >= np;
+        const bool do_rescale = i > 0 && __any_sync(HS_FULL_MASK, corr != 1.f);
+        if (do_gather || do_rescale) {
             mbar_wait(bar_pv, (unsigned int)(i - 1) & 1u, p.err);
             tc_fence_after_sync();
-            const int nx = i - 1 + UM_STAGES;                // its stage is free again: a tree tile is gathered here,
-            if (nx < ntiles && nx >= np) gather_tree(nx);    // a prefix tile is requested by the issuing thread
         }
-        // O in tensor memory is rescaled only if some row of this warp needs it (the load/store are warp-wide);
-        // each of a row's two threads rescales its 64 of the 128 columns
-        if (i > 0 && __any_sync(HS_FULL_MASK, corr != 1.f)) {
+        if (do_gather) gather_tree(nx);                      // (a prefix tile is requested by the issuing thread)
+        if (do_rescale) {
 #pragma unroll 1
             for (int ch = 0; ch < 2; ++ch) {
                 unsigned int ov[32];
@@ -658,25 +682,17 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
             }
             tmem_wait_st();
         }
-        float lsum = 0.f;
 #pragma unroll
-        for (int c8 = 0; c8 < 4; ++c8) {
-            float pv[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                pv[e] = ex2_approx(__uint_as_float(sr[c8 * 8 + e]) - muse);
-                lsum += pv[e];
-            }
-            uint4 pk;
-            pk.x = pack_bf16(pv[0], pv[1]); pk.y = pack_bf16(pv[2], pv[3]);
-            pk.z = pack_bf16(pv[4], pv[5]); pk.w = pack_bf16(pv[6], pv[7]);
-            *reinterpret_cast<uint4*>(gP + row * 128 + (((half * 4 + c8) ^ (row & 7)) << 4)) = pk;
-        }
+        for (int c8 = 0; c8 < 4; ++c8)
+            *reinterpret_cast<uint4*>(gP + (i & 1) * UM_P_BYTES + row * 128 + (((half * 4 + c8) ^ (row & 7)) << 4)) = pk[c8];
         lrun = fmaf(lrun, corr, lsum);                       // the sum over this thread's half of the columns
         fence_proxy_async_smem();                            // P (and gathered tree tiles) -> tensor cores
         tc_fence_before_sync();
         mbar_arrive(bar_p);
     }
+    // A parity wait names the current or the preceding phase only; a softmax thread that skipped waits knows no more
+    // than that O += P V of tile ntiles - 3 is complete, so the last two phases are waited for in order.
+    if (ntiles > 1 && warp < 8) mbar_wait(bar_pv, (unsigned int)(ntiles - 2) & 1u, p.err);
     if (ntiles > 0 && warp < 8) mbar_wait(bar_pv, (unsigned int)(ntiles - 1) & 1u, p.err);
     __syncwarp();                                        // the issuing warp reconverges (warp-aligned barriers follow)
     tc_fence_after_sync();
@@ -720,7 +736,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         const unsigned int s_recv = smem_base, s_stage = smem_base + UM_RECV_BYTES;
         const int rows_max = (ATT_BM + ns - 1) / ns + 1;
         const int r_lo = (split * ATT_BM + ns - 1) / ns, r_hi = ((split + 1) * ATT_BM + ns - 1) / ns;   // rows this CTA owns
-        long long* s_og = reinterpret_cast<long long*>(gP);                          // output row of each owned row (or -1)
+        long long* s_og = reinterpret_cast<long long*>(gP);               // (P buffers are idle now)                          // output row of each owned row (or -1)
         if (tid == 0) mbar_expect_tx(bar_r, (unsigned int)(ns * (r_hi - r_lo) * ATT_PO_STRIDE * 4));
         if (tid < r_hi - r_lo) {
             const int rg = m0 + r_lo + tid;
