@@ -408,19 +408,22 @@ tree_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, co
 
 // =====================================================================================================
 // tcgen05 version: S = Q K^T and O += P V by the 5th-generation tensor cores, accumulators in tensor
-// memory.  128 threads; thread t owns query row t of the block (= tensor-memory lane t), so the
-// softmax needs no shuffles.  Per 64-key tile: thread 0 has issued S = Q K^T (8 instructions of
-// K = 16, operands straight from the swizzled TMA tiles: Q and K are K-major) and committed to an
-// mbarrier; every thread waits, loads its row of S from tensor memory, masks, exponentiates, writes
-// its row of P (bf16) to a swizzled shared-memory tile; after a barrier thread 0 issues O += P V
-// (V is the MN-major operand, the same swizzled tile as it arrived by TMA) and S of the next tile.
-// O is rescaled in tensor memory only when a row's running maximum grows.
+// memory.  Two softmax warpgroups run two independent online-softmax streams over the block's 128 query
+// rows: warpgroup g takes the KV tiles i = g, g + 2, ... and keeps its own S buffer, P buffer, running
+// (max, sum) and O accumulator; thread t of a warpgroup owns query row t (= tensor-memory lane t), so the
+// softmax needs no shuffles and the two streams never wait for one another: while one exponentiates (the
+// special-function unit), the other loads, masks and stores.  A ninth warp's first thread issues all
+// tensor-core and TMA work: S = Q K^T two tiles ahead (8 instructions of K = 16, operands straight from
+// the swizzled TMA tiles: Q and K are K-major), O_g += P V as soon as a P is written (V is the MN-major
+// operand, the same swizzled tile as it arrived by TMA), stage refills once a tile's P V is complete.
+// A stream rescales its O in tensor memory only when a row's running maximum grows.  After the last
+// tile the two streams are combined like two splits, in registers.
 // =====================================================================================================
-#define UM_THREADS 288                               // eight softmax warps (two threads per query row) + the issuing warp
+#define UM_THREADS 288                               // two softmax warpgroups + the issuing warp
 #define UM_ROWS_THREADS 128
-#define UM_SM_THREADS 256                            // softmax threads: row = tid & 127, column half = tid >> 7
+#define UM_SM_THREADS 256                            // softmax threads: row = tid & 127, stream = tid >> 7
 #define UM_P_BYTES (ATT_BM * ATT_BN * 2)             // 16 KiB: P tile, 128 rows x 64 keys bf16
-#define UM_TMEM_COLS 256                             // S (two buffers): columns 0..127, O: columns 128..255
+#define UM_TMEM_COLS 512                             // S of stream g: columns 64 g ..; O of stream g: columns 128 + 128 g ..
 #define UM_STAGES 4
 #define UM_RECV_BYTES (76 * 1024)                    // after the tile loop: partials pushed by the splits of the cluster
 #define UM_SMEM_BYTES (UM_STAGES * ATT_STAGE_BYTES + ATT_Q_BYTES + 2 * UM_P_BYTES + 4096 + 1024)
@@ -438,14 +441,15 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const unsigned int sQ = smem_base + UM_STAGES * ATT_STAGE_BYTES;
     const unsigned int sP = sQ + ATT_Q_BYTES;
-    const unsigned int bar0 = sP + 2 * UM_P_BYTES;   // (P is double-buffered) full[UM_STAGES], S-ready[2], PV-done, partials-received, P-written, tensor-memory base
-    const unsigned int bar_s = bar0 + UM_STAGES * 8, bar_pv = bar_s + 16, bar_r = bar_pv + 8, bar_p = bar_r + 8,
-                       tslot = bar_p + 8;
+    // barriers: full[UM_STAGES], S-ready[2], PV-done, partials-received, all-MMAs-done, P-written[2]; tensor-memory base
+    const unsigned int bar0 = sP + 2 * UM_P_BYTES;
+    const unsigned int bar_s = bar0 + UM_STAGES * 8, bar_pv = bar_s + 16, bar_r = bar_pv + 8, bar_done = bar_r + 8,
+                       bar_p = bar_done + 8, tslot = bar_p + 16;
     unsigned char* gQ = smem_gen + UM_STAGES * ATT_STAGE_BYTES;
     unsigned char* gP = gQ + ATT_Q_BYTES;
-    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + 2 * UM_P_BYTES + (UM_STAGES + 5) * 8);
-    float* s_xch = reinterpret_cast<float*>(gP + 2 * UM_P_BYTES + 1024);      // [2][2][128]: half-row maxima (per S buffer)
-    float* s_lx = s_xch + 4 * ATT_BM;                                    // [2][128]: half-row sums at the end
+    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + 2 * UM_P_BYTES + (UM_STAGES + 7) * 8);
+    float* s_mx = reinterpret_cast<float*>(gP + 2 * UM_P_BYTES + 1024);      // [2][128]: the streams' row maxima at the end
+    float* s_lx = s_mx + 2 * ATT_BM;                                     // [2][128]: the streams' row sums
 
     // ---- before the dependency wait: barriers, tensor memory, the first KV prefix tiles -----------------
     const int kv0 = p.kv_off[b];
@@ -473,8 +477,9 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     };
     const int pre = min(np, UM_STAGES);
     if (tid == 0) {
-        for (int i = 0; i < UM_STAGES + 4; ++i) mbar_init(bar0 + i * 8, 1);
-        mbar_init(bar_p, UM_SM_THREADS);                 // P of a tile is written: one arrival per softmax thread
+        for (int i = 0; i < UM_STAGES + 5; ++i) mbar_init(bar0 + i * 8, 1);
+        mbar_init(bar_p, UM_ROWS_THREADS);               // P of a tile is written: one arrival per thread of the stream
+        mbar_init(bar_p + 8, UM_ROWS_THREADS);
         mbar_init_fence();
         for (int i = 0; i < pre; ++i) issue_prefix(i);
     }
@@ -489,8 +494,8 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     tc_fence_after_sync();
     const unsigned int tmem_base = *tslot_gen;
     const unsigned int lane_off = (unsigned int)((warp & 3) * 32) << 16;   // a warp reaches lanes 32 * (warp % 4) ...
-    const int row = tid & (ATT_BM - 1), half = (tid >> 7) & 1;               // the thread's query row and column half
-    const unsigned int tS = tmem_base, tO = tmem_base + 128;
+    const int row = tid & (ATT_BM - 1), half = (tid >> 7) & 1;               // the thread's query row and stream
+    const unsigned int tS = tmem_base, tO = tmem_base + 128;                 // (+ 64 / + 128 columns for stream 1)
 
     const int nk = (p.status[b] == 0) ? p.n_keep[b] : 0;
     const int M = nk * p.G;
@@ -505,9 +510,9 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     const int nt_tree = (split == p.nsplit - 1) ? (nk + ATT_BN - 1) / ATT_BN : 0;
     const int ntiles = np + nt_tree;
 
-    // tree keys/values: gathered rows, 16-byte loads (all of a thread's loads in flight together), swizzled
-    // stores; 2 x 1024 chunks / 256 threads
-    auto gather_tree = [&](int i) {
+    // tree keys/values: gathered rows, 16-byte loads (four of a thread's loads in flight together), swizzled
+    // stores; 2 x 1024 chunks by nthr threads (thread t of them), chunks t + (it0 .. it0 + 3) * nthr
+    auto gather_tree = [&](int i, int t, int nthr, int it0) {
         unsigned char* gK = smem_gen + (i % UM_STAGES) * ATT_STAGE_BYTES;
         unsigned char* gV = gK + ATT_TILE_BYTES;
         const int j0 = (i - np) * ATT_BN;
@@ -515,7 +520,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         int trow[4];
 #pragma unroll
         for (int it = 0; it < 4; ++it) {
-            const int j = j0 + ((tid + it * UM_SM_THREADS) >> 4);
+            const int j = j0 + ((t + (it0 + it) * nthr) >> 4);
             trow[it] = -1;
             if (j < nk) trow[it] = (p.layout == HS_ROWS_ORIGINAL) ? p.node_off[b] + p.keep_idx[koff + j] : koff + j;
         }
@@ -524,14 +529,14 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
             kvv[it] = make_uint4(0, 0, 0, 0);
             vvv[it] = make_uint4(0, 0, 0, 0);
             if (trow[it] >= 0) {
-                const size_t off = ((size_t)trow[it] * p.hkv + h) * HS_HEAD_DIM + (tid & 15) * 8;
+                const size_t off = ((size_t)trow[it] * p.hkv + h) * HS_HEAD_DIM + (t & 15) * 8;
                 kvv[it] = __ldg(reinterpret_cast<const uint4*>(p.k_tree + off));
                 vvv[it] = __ldg(reinterpret_cast<const uint4*>(p.v_tree + off));
             }
         }
 #pragma unroll
         for (int it = 0; it < 4; ++it) {
-            const int c = tid + it * UM_SM_THREADS;
+            const int c = t + (it0 + it) * nthr;
             *reinterpret_cast<uint4*>(gK + tile_off(c >> 4, c & 15)) = kvv[it];
             *reinterpret_cast<uint4*>(gV + tile_off(c >> 4, c & 15)) = vvv[it];
         }
@@ -561,7 +566,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         }
     }
     if (warp < 8)
-        for (int i = np; i < min(ntiles, UM_STAGES); ++i) gather_tree(i);  // tree tiles that open the pipeline
+        for (int i = np; i < min(ntiles, UM_STAGES); ++i) gather_tree(i, tid, UM_SM_THREADS, 0);  // tree tiles that open the pipeline
     fence_proxy_async_smem();                        // generic stores -> visible to the tensor cores
     __syncthreads();
 
@@ -595,23 +600,28 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
                 mbar_wait(bar_pv, (unsigned int)(i - 1) & 1u, p.err);
                 issue_prefix(i - 1 + UM_STAGES);
             }
-            mbar_wait(bar_p, (unsigned int)i & 1u, p.err);   // P of tile i is in shared memory, S buffer i & 1 is read
+            mbar_wait(bar_p + (i & 1) * 8, (unsigned int)(i >> 1) & 1u, p.err);   // P of tile i is written, its S is read
             tc_fence_after_sync();
             const unsigned int sV = smem_base + (i % UM_STAGES) * ATT_STAGE_BYTES + ATT_TILE_BYTES;
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)                   // 16 keys per instruction: two 8-key groups of V
-                umma_ss_bf16(tO, umma_desc_sw128(sP + (i & 1) * UM_P_BYTES + kk * 32, 16, 1024),
-                             umma_desc_sw128(sV + kk * 2048, ATT_TILE_BYTES / 2, 1024), idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
+                umma_ss_bf16(tO + (i & 1) * HS_HEAD_DIM, umma_desc_sw128(sP + (i & 1) * UM_P_BYTES + kk * 32, 16, 1024),
+                             umma_desc_sw128(sV + kk * 2048, ATT_TILE_BYTES / 2, 1024), idesc_pv, (i > 1 || kk > 0) ? 1u : 0u);
             umma_commit(bar_pv);
             if (i + 2 < ntiles) issue_qk(i + 2);
         }
+        if (ntiles > 0) umma_commit(bar_done);               // every tensor-core operation of this CTA is complete
     }
+    // Stream `half`: tiles half, half + 2, ...  What a stream touches at tile i (its S and P buffers, its O) was
+    // last used by the tensor cores for tile i - 2, and S of tile i was committed after O += P V of tile i - 2 was
+    // issued: once S is there, nothing else has to be waited for.
 #pragma unroll 1
-    for (int i = 0; i < ntiles && warp < 8; ++i) {
-        mbar_wait(bar_s + (i & 1) * 8, (unsigned int)(i >> 1) & 1u, p.err);      // S of tile i is complete
+    for (int i = half; i < ntiles && warp < 8; i += 2) {
+        mbar_wait(bar_s + half * 8, (unsigned int)(i >> 1) & 1u, p.err);         // S of tile i is complete
         tc_fence_after_sync();
-        unsigned int sr[32];                                 // this thread's 32 of the row's 64 scores
-        tmem_ld32(tS + (i & 1) * ATT_BN + half * 32 + lane_off, sr);
+        unsigned int sr[64];                                 // the row's 64 scores
+        tmem_ld32(tS + half * ATT_BN + lane_off, sr);
+        tmem_ld32(tS + half * ATT_BN + 32 + lane_off, sr + 32);
         tmem_wait_ld();
 
         const bool is_tree = i >= np;
@@ -619,87 +629,100 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         const int nvis = (is_tree ? nk : L) - col0;          // columns of this tile inside the sequence / tree
         // The scores stay unscaled in registers (the scale is positive: it commutes with the maximum and folds into
         // the exponent's multiply-add). A prefix tile inside the sequence needs no mask at all.
-        float mx = -CUDART_INF_F;
-        if (!is_tree && nvis >= ATT_BN) {
-#pragma unroll
-            for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(sr[c]));
-        } else {
+        float mxa = -CUDART_INF_F, mxb = -CUDART_INF_F;
+        if (is_tree || nvis < ATT_BN) {
             // a tree tile of 64 keys lies inside one 64-bit word of the ancestor mask
             unsigned long long vis64 = nvis >= 64 ? ~0ull : ((1ull << max(nvis, 0)) - 1ull);
             if (is_tree) vis64 &= (col0 == 0 ? mk0 : mk1);
-            const unsigned int vis = (unsigned int)(vis64 >> (half * 32));
+            const unsigned int vlo = (unsigned int)vis64, vhi = (unsigned int)(vis64 >> 32);
 #pragma unroll
             for (int c = 0; c < 32; ++c) {
-                if (!((vis >> c) & 1u)) sr[c] = __float_as_uint(-CUDART_INF_F);
-                mx = fmaxf(mx, __uint_as_float(sr[c]));
+                if (!((vlo >> c) & 1u)) sr[c] = __float_as_uint(-CUDART_INF_F);
+                if (!((vhi >> c) & 1u)) sr[32 + c] = __float_as_uint(-CUDART_INF_F);
             }
         }
-        mx *= p.scale_log2;
-        // the row maximum of this tile: exchanged between the two threads of a row (one buffer per S buffer)
-        float* xch = s_xch + (i & 1) * 2 * ATT_BM;
-        xch[half * ATT_BM + row] = mx;
-        asm volatile("bar.sync 1, %0;" ::"n"(UM_SM_THREADS) : "memory");
-        mx = fmaxf(mx, xch[(half ^ 1) * ATT_BM + row]);
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+            mxa = fmaxf(mxa, __uint_as_float(sr[c]));
+            mxb = fmaxf(mxb, __uint_as_float(sr[32 + c]));
+        }
+        const float mx = fmaxf(mxa, mxb) * p.scale_log2;
         const float mnew = fmaxf(mrun, mx);
         const float muse = (mnew == -CUDART_INF_F) ? 0.f : mnew;
-        const float corr = ex2_approx(mrun - muse);          // 1 when the maximum did not grow, 0 at the first tile
+        const float corr = ex2_approx(mrun - muse);          // 1 when the maximum did not grow, 0 at the stream's first tile
         mrun = mnew;
-        // the row's P of this tile, in registers first: nothing has been waited for so far
-        float lsum = 0.f;
-        uint4 pk[4];
+        // the row's P of this tile, in registers first
+        float lsa = 0.f, lsb = 0.f;
+        uint4 pk[8];
 #pragma unroll
-        for (int c8 = 0; c8 < 4; ++c8) {
+        for (int c8 = 0; c8 < 8; ++c8) {
             float pv[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                pv[e] = ex2_approx(fmaf(__uint_as_float(sr[c8 * 8 + e]), p.scale_log2, -muse));
-                lsum += pv[e];
-            }
+            for (int e = 0; e < 8; ++e) pv[e] = ex2_approx(fmaf(__uint_as_float(sr[c8 * 8 + e]), p.scale_log2, -muse));
+            lsa += (pv[0] + pv[1]) + (pv[2] + pv[3]);
+            lsb += (pv[4] + pv[5]) + (pv[6] + pv[7]);
             pk[c8].x = pack_bf16(pv[0], pv[1]); pk[c8].y = pack_bf16(pv[2], pv[3]);
             pk[c8].z = pack_bf16(pv[4], pv[5]); pk[c8].w = pack_bf16(pv[6], pv[7]);
         }
-        // O and the stage of tile i - 1 may be touched only when O += P V of tile i - 1 is complete; that is
-        // needed when a tree tile is gathered into the stage or when O has to be rescaled (the load/store are
-        // warp-wide: a warp rescales if any of its rows needs it; each of a row's two threads does 64 columns).
-        // P itself is double-buffered: buffer i & 1 was last read by tile i - 2, complete since S of tile i is.
+        lrun = fmaf(lrun, corr, lsa + lsb);
+        // A tree tile is gathered into the stage of tile i - 1 once that tile's O += P V is complete (a prefix tile
+        // is requested by the issuing thread).  S of tile i says that P V of tile i - 2 is complete and P of tile i
+        // is not written yet, so the barrier is in phase i - 1 or i: the parity wait is unambiguous.
         const int nx = i - 1 + UM_STAGES;
-        const bool do_gather = i >= 1 && nx < ntiles && nx >= np;
-        const bool do_rescale = i > 0 && __any_sync(HS_FULL_MASK, corr != 1.f);
-        if (do_gather || do_rescale) {
+        if (i >= 1 && nx < ntiles && nx >= np) {
             mbar_wait(bar_pv, (unsigned int)(i - 1) & 1u, p.err);
-            tc_fence_after_sync();
+            gather_tree(nx, row, UM_ROWS_THREADS, 0);
+            gather_tree(nx, row, UM_ROWS_THREADS, 4);
         }
-        if (do_gather) gather_tree(nx);                      // (a prefix tile is requested by the issuing thread)
-        if (do_rescale) {
+        // rescale this stream's O (the load/store are warp-wide: a warp rescales if any of its rows needs it)
+        if (i >= 2 && __any_sync(HS_FULL_MASK, corr != 1.f)) {
 #pragma unroll 1
-            for (int ch = 0; ch < 2; ++ch) {
+            for (int ch = 0; ch < 4; ++ch) {
                 unsigned int ov[32];
-                tmem_ld32(tO + lane_off + half * 64 + ch * 32, ov);
+                tmem_ld32(tO + half * HS_HEAD_DIM + lane_off + ch * 32, ov);
                 tmem_wait_ld();
 #pragma unroll
                 for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * corr);
-                tmem_st32(tO + lane_off + half * 64 + ch * 32, ov);
+                tmem_st32(tO + half * HS_HEAD_DIM + lane_off + ch * 32, ov);
             }
             tmem_wait_st();
         }
 #pragma unroll
-        for (int c8 = 0; c8 < 4; ++c8)
-            *reinterpret_cast<uint4*>(gP + (i & 1) * UM_P_BYTES + row * 128 + (((half * 4 + c8) ^ (row & 7)) << 4)) = pk[c8];
-        lrun = fmaf(lrun, corr, lsum);                       // the sum over this thread's half of the columns
+        for (int c8 = 0; c8 < 8; ++c8)
+            *reinterpret_cast<uint4*>(gP + half * UM_P_BYTES + row * 128 + ((c8 ^ (row & 7)) << 4)) = pk[c8];
         fence_proxy_async_smem();                            // P (and gathered tree tiles) -> tensor cores
         tc_fence_before_sync();
-        mbar_arrive(bar_p);
+        mbar_arrive(bar_p + half * 8);
     }
-    // A parity wait names the current or the preceding phase only; a softmax thread that skipped waits knows no more
-    // than that O += P V of tile ntiles - 3 is complete, so the last two phases are waited for in order.
-    if (ntiles > 1 && warp < 8) mbar_wait(bar_pv, (unsigned int)(ntiles - 2) & 1u, p.err);
-    if (ntiles > 0 && warp < 8) mbar_wait(bar_pv, (unsigned int)(ntiles - 1) & 1u, p.err);
+    if (ntiles > 0 && warp < 8) mbar_wait(bar_done, 0u, p.err);
     __syncwarp();                                        // the issuing warp reconverges (warp-aligned barriers follow)
     tc_fence_after_sync();
-    // the row sum: both halves together
-    if (warp < 8) s_lx[half * ATT_BM + row] = lrun;
+    // the two streams of a row are combined like two splits: weights w0, w1 on the streams' O, one (max, sum)
+    if (warp < 8) { s_mx[half * ATT_BM + row] = mrun; s_lx[half * ATT_BM + row] = lrun; }
     __syncthreads();
-    if (warp < 8) lrun += s_lx[(half ^ 1) * ATT_BM + row];
+    float w0 = 0.f, w1 = 0.f;
+    if (warp < 8) {
+        const float m_a = s_mx[row], m_b = s_mx[ATT_BM + row];
+        mrun = fmaxf(m_a, m_b);
+        const float muse = (mrun == -CUDART_INF_F) ? 0.f : mrun;
+        w0 = ex2_approx(m_a - muse);
+        w1 = ex2_approx(m_b - muse);
+        lrun = s_lx[row] * w0 + s_lx[ATT_BM + row] * w1;
+    }
+    // this thread's 32 columns [half * 64 + ch * 32, + 32) of the row's combined O (a stream without tiles has no O)
+    auto load_o = [&](int ch, unsigned int* ov) {
+        unsigned int oa[32], ob[32];
+        if (ntiles > 0) tmem_ld32(tO + lane_off + half * 64 + ch * 32, oa);
+        if (ntiles > 1) tmem_ld32(tO + HS_HEAD_DIM + lane_off + half * 64 + ch * 32, ob);
+        tmem_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+            float v = 0.f;
+            if (ntiles > 0) v = __uint_as_float(oa[c]) * w0;
+            if (ntiles > 1) v = fmaf(__uint_as_float(ob[c]), w1, v);
+            ov[c] = __float_as_uint(v);
+        }
+    };
 
     // ---- epilogue ----------------------------------------------------------------------------------------------
     if (p.nsplit == 1) {
@@ -707,8 +730,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
 #pragma unroll 1
         for (int ch = 0; ch < 2 && warp < 8; ++ch) {
             unsigned int ov[32];
-            tmem_ld32(tO + lane_off + half * 64 + ch * 32, ov);
-            tmem_wait_ld();
+            load_o(ch, ov);
             if (orow >= 0) {
                 uint4* dst = reinterpret_cast<uint4*>(p.out + (size_t)orow * HS_HEAD_DIM + half * 64 + ch * 32);
 #pragma unroll
@@ -751,11 +773,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
 #pragma unroll 1
         for (int ch = 0; ch < 2 && warp < 8; ++ch) {
             unsigned int ov[32];
-            if (ntiles > 0) { tmem_ld32(tO + lane_off + half * 64 + ch * 32, ov); tmem_wait_ld(); }
-            else {
-#pragma unroll
-                for (int c = 0; c < 32; ++c) ov[c] = 0u;
-            }
+            load_o(ch, ov);
             float4* dst = reinterpret_cast<float4*>(stage_po + row * ATT_PO_STRIDE + half * 64 + ch * 32);
 #pragma unroll
             for (int q = 0; q < 8; ++q)
