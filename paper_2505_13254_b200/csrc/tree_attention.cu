@@ -441,13 +441,16 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const unsigned int sQ = smem_base + UM_STAGES * ATT_STAGE_BYTES;
     const unsigned int sP = sQ + ATT_Q_BYTES;
-    // barriers: full[UM_STAGES], S-ready[2], PV-done, partials-received, all-MMAs-done, P-written[2]; tensor-memory base
-    const unsigned int bar0 = sP + 2 * UM_P_BYTES;
-    const unsigned int bar_s = bar0 + UM_STAGES * 8, bar_pv = bar_s + 16, bar_r = bar_pv + 8, bar_done = bar_r + 8,
+    // barriers: K-full[UM_STAGES], V-full[UM_STAGES], S-ready[2], PV-done[2], partials-received, all-MMAs-done,
+    // P-written[2]; then the tensor-memory base.  S-ready, PV-done and P-written alternate with the tile's parity: a
+    // parity wait can only tell the current phase from the one before, and with two barriers the thread that waits
+    // for tile i is never more than one completion behind (the next completion on the same barrier is tile i + 2's).
+    const unsigned int bar0 = sP + 2 * UM_P_BYTES, bar_v = bar0 + UM_STAGES * 8;
+    const unsigned int bar_s = bar_v + UM_STAGES * 8, bar_pv = bar_s + 16, bar_r = bar_pv + 16, bar_done = bar_r + 8,
                        bar_p = bar_done + 8, tslot = bar_p + 16;
     unsigned char* gQ = smem_gen + UM_STAGES * ATT_STAGE_BYTES;
     unsigned char* gP = gQ + ATT_Q_BYTES;
-    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + 2 * UM_P_BYTES + (UM_STAGES + 7) * 8);
+    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + 2 * UM_P_BYTES + (2 * UM_STAGES + 8) * 8);
     float* s_mx = reinterpret_cast<float*>(gP + 2 * UM_P_BYTES + 1024);      // [2][128]: the streams' row maxima at the end
     float* s_lx = s_mx + 2 * ATT_BM;                                     // [2][128]: the streams' row sums
 
@@ -457,31 +460,30 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     int t_prefix, t0, t1;
     prefix_range(L, p.nsplit, split, t_prefix, t0, t1);
     const int np = t1 - t0;
-    auto issue_prefix = [&](int i) {                 // thread 0: tile i of this CTA into stage i % UM_STAGES
+    // one thread: K (V) of prefix tile i of this CTA into stage i % UM_STAGES; K and V complete on barriers of their own,
+    // because a stage's K is free again (after S = Q K^T) two tiles before its V is (after O += P V)
+    auto issue_kv = [&](int i, bool is_v) {
         const int stage = i % UM_STAGES;
-        const unsigned int sK = smem_base + stage * ATT_STAGE_BYTES, sV = sK + ATT_TILE_BYTES;
-        const unsigned int bar = bar0 + stage * 8;
+        const unsigned int dst = smem_base + stage * ATT_STAGE_BYTES + (is_v ? ATT_TILE_BYTES : 0);
+        const unsigned int bar = (is_v ? bar_v : bar0) + stage * 8;
+        const CUtensorMap* tm = is_v ? &tmV : &tmK;
         const int tok = kv0 + (t0 + i) * ATT_BN;
-        mbar_expect_tx(bar, ATT_STAGE_BYTES);
+        mbar_expect_tx(bar, ATT_TILE_BYTES);
         if (p.head_first) {
-            tma_load_3d(sK, &tmK, 0, tok, h, bar);
-            tma_load_3d(sK + ATT_TILE_BYTES / 2, &tmK, 64, tok, h, bar);
-            tma_load_3d(sV, &tmV, 0, tok, h, bar);
-            tma_load_3d(sV + ATT_TILE_BYTES / 2, &tmV, 64, tok, h, bar);
+            tma_load_3d(dst, tm, 0, tok, h, bar);
+            tma_load_3d(dst + ATT_TILE_BYTES / 2, tm, 64, tok, h, bar);
         } else {
-            tma_load_3d(sK, &tmK, 0, h, tok, bar);
-            tma_load_3d(sK + ATT_TILE_BYTES / 2, &tmK, 64, h, tok, bar);
-            tma_load_3d(sV, &tmV, 0, h, tok, bar);
-            tma_load_3d(sV + ATT_TILE_BYTES / 2, &tmV, 64, h, tok, bar);
+            tma_load_3d(dst, tm, 0, h, tok, bar);
+            tma_load_3d(dst + ATT_TILE_BYTES / 2, tm, 64, h, tok, bar);
         }
     };
     const int pre = min(np, UM_STAGES);
     if (tid == 0) {
-        for (int i = 0; i < UM_STAGES + 5; ++i) mbar_init(bar0 + i * 8, 1);
+        for (int i = 0; i < 2 * UM_STAGES + 6; ++i) mbar_init(bar0 + i * 8, 1);
         mbar_init(bar_p, UM_ROWS_THREADS);               // P of a tile is written: one arrival per thread of the stream
         mbar_init(bar_p + 8, UM_ROWS_THREADS);
         mbar_init_fence();
-        for (int i = 0; i < pre; ++i) issue_prefix(i);
+        for (int i = 0; i < pre; ++i) { issue_kv(i, false); issue_kv(i, true); }
     }
     if (warp == 0) {
         tmem_alloc(tslot, UM_TMEM_COLS);
@@ -501,7 +503,10 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     const int M = nk * p.G;
     if (m0 >= M) {                                   // nothing to do (the same for every CTA of the cluster)
         if (tid == 0)
-            for (int i = 0; i < pre; ++i) mbar_wait(bar0 + i * 8, 0u, p.err);   // no copy may outlive the CTA
+            for (int i = 0; i < pre; ++i) {              // no copy may outlive the CTA
+                mbar_wait(bar0 + i * 8, 0u, p.err);
+                mbar_wait(bar_v + i * 8, 0u, p.err);
+            }
         __syncthreads();
         if (warp == 0) tmem_dealloc(tmem_base, UM_TMEM_COLS);
         return;
@@ -572,43 +577,61 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
 
     const unsigned int idesc_qk = umma_idesc_bf16(ATT_BM, ATT_BN, false);
     const unsigned int idesc_pv = umma_idesc_bf16(ATT_BM, HS_HEAD_DIM, true);
-    // thread 0: S = Q K^T of tile i into S buffer i & 1 (waits for the tile if it comes by TMA), then commit
+    // Operand descriptors: the start-address field (16-byte units, low 14 bits) is the only part that varies, and no
+    // shared-memory address reaches 2^18, so an offset is added to a descriptor built once.
+    const unsigned long long dq0 = umma_desc_sw128(sQ, 16, 1024), dk0 = umma_desc_sw128(smem_base, 16, 1024);
+    const unsigned long long dp0 = umma_desc_sw128(sP, 16, 1024),
+                             dv0 = umma_desc_sw128(smem_base + ATT_TILE_BYTES, ATT_TILE_BYTES / 2, 1024);
+    // the issuing thread: S = Q K^T of tile i into S buffer i & 1 (waits for K if it comes by TMA), then commit
     auto issue_qk = [&](int i) {
         const int stage = i % UM_STAGES;
         if (i < np) mbar_wait(bar0 + stage * 8, (unsigned int)(i / UM_STAGES) & 1u, p.err);
         tc_fence_after_sync();
-        const unsigned int sK = smem_base + stage * ATT_STAGE_BYTES;
+        const unsigned long long dk = dk0 + (unsigned long long)(stage * (ATT_STAGE_BYTES >> 4));
+        const unsigned int ts = tS + (i & 1) * ATT_BN;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
             const unsigned int koffb = (ks >> 2) * (ATT_TILE_BYTES / 2) + (ks & 3) * 32;
             const unsigned int qoffb = (ks >> 2) * (ATT_Q_BYTES / 2) + (ks & 3) * 32;
-            umma_ss_bf16(tS + (i & 1) * ATT_BN, umma_desc_sw128(sQ + qoffb, 16, 1024), umma_desc_sw128(sK + koffb, 16, 1024),
-                         idesc_qk, ks > 0 ? 1u : 0u);
+            umma_ss_bf16(ts, dq0 + (qoffb >> 4), dk + (koffb >> 4), idesc_qk, ks > 0 ? 1u : 0u);
         }
         umma_commit(bar_s + (i & 1) * 8);
+    };
+    // O of stream i & 1 += P V of tile i (waits for V if it comes by TMA), then commit
+    auto issue_pv = [&](int i) {
+        const int stage = i % UM_STAGES;
+        if (i < np) mbar_wait(bar_v + stage * 8, (unsigned int)(i / UM_STAGES) & 1u, p.err);
+        tc_fence_after_sync();
+        const unsigned long long dv = dv0 + (unsigned long long)(stage * (ATT_STAGE_BYTES >> 4));
+        const unsigned long long dp = dp0 + (unsigned long long)((i & 1) * (UM_P_BYTES >> 4));
+        const unsigned int to = tO + (i & 1) * HS_HEAD_DIM;
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)                       // 16 keys per instruction: two 8-key groups of V
+            umma_ss_bf16(to, dp + (kk * 32 >> 4), dv + (kk * 2048 >> 4), idesc_pv, (i > 1 || kk > 0) ? 1u : 0u);
+        umma_commit(bar_pv + (i & 1) * 8);
     };
     float mrun = -CUDART_INF_F, lrun = 0.f;
 
     // ---- KV tiles ------------------------------------------------------------------------------------------
     if (tid == UM_SM_THREADS) {
-        // The issuing thread: S two tiles ahead of the softmax, O += P V as soon as a P is written, TMA refills.
+        // The issuing thread: S two tiles ahead of the softmax, O += P V as soon as a P is written; refills: K of
+        // tile i + 4 (S of tile i is long complete; waited for before S of tile i + 2 is committed to the same
+        // barrier) and V of tile i + 3 (once O += P V of tile i - 1 is complete).
         if (ntiles > 0) issue_qk(0);
         if (ntiles > 1) issue_qk(1);
 #pragma unroll 1
         for (int i = 0; i < ntiles; ++i) {
-            if (i >= 1 && i - 1 + UM_STAGES < np) {          // the stage of tile i - 1 is free once its P V is done
-                mbar_wait(bar_pv, (unsigned int)(i - 1) & 1u, p.err);
-                issue_prefix(i - 1 + UM_STAGES);
-            }
             mbar_wait(bar_p + (i & 1) * 8, (unsigned int)(i >> 1) & 1u, p.err);   // P of tile i is written, its S is read
-            tc_fence_after_sync();
-            const unsigned int sV = smem_base + (i % UM_STAGES) * ATT_STAGE_BYTES + ATT_TILE_BYTES;
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk)                   // 16 keys per instruction: two 8-key groups of V
-                umma_ss_bf16(tO + (i & 1) * HS_HEAD_DIM, umma_desc_sw128(sP + (i & 1) * UM_P_BYTES + kk * 32, 16, 1024),
-                             umma_desc_sw128(sV + kk * 2048, ATT_TILE_BYTES / 2, 1024), idesc_pv, (i > 1 || kk > 0) ? 1u : 0u);
-            umma_commit(bar_pv);
+            issue_pv(i);
+            if (i + UM_STAGES < np) {                        // S of tile i is complete (it was read): K's stage is free
+                mbar_wait(bar_s + (i & 1) * 8, (unsigned int)(i >> 1) & 1u, p.err);
+                issue_kv(i + UM_STAGES, false);
+            }
             if (i + 2 < ntiles) issue_qk(i + 2);
+            if (i >= 1 && i - 1 + UM_STAGES < np) {          // V's stage of tile i - 1 is free once its P V is done
+                mbar_wait(bar_pv + ((i - 1) & 1) * 8, (unsigned int)((i - 1) >> 1) & 1u, p.err);
+                issue_kv(i - 1 + UM_STAGES, true);
+            }
         }
         if (ntiles > 0) umma_commit(bar_done);               // every tensor-core operation of this CTA is complete
     }
@@ -666,11 +689,11 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         }
         lrun = fmaf(lrun, corr, lsa + lsb);
         // A tree tile is gathered into the stage of tile i - 1 once that tile's O += P V is complete (a prefix tile
-        // is requested by the issuing thread).  S of tile i says that P V of tile i - 2 is complete and P of tile i
-        // is not written yet, so the barrier is in phase i - 1 or i: the parity wait is unambiguous.
+        // is requested by the issuing thread).  P of tile i + 1 is not written before this stream's P of tile i is,
+        // so the barrier of tile i - 1's parity cannot be a phase ahead: the parity wait is unambiguous.
         const int nx = i - 1 + UM_STAGES;
         if (i >= 1 && nx < ntiles && nx >= np) {
-            mbar_wait(bar_pv, (unsigned int)(i - 1) & 1u, p.err);
+            mbar_wait(bar_pv + ((i - 1) & 1) * 8, (unsigned int)((i - 1) >> 1) & 1u, p.err);
             gather_tree(nx, row, UM_ROWS_THREADS, 0);
             gather_tree(nx, row, UM_ROWS_THREADS, 4);
         }
