@@ -412,14 +412,15 @@ tree_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, co
 // rows: warpgroup g takes the KV tiles i = g, g + 2, ... and keeps its own S buffer, P buffer, running
 // (max, sum) and O accumulator; thread t of a warpgroup owns query row t (= tensor-memory lane t), so the
 // softmax needs no shuffles and the two streams never wait for one another: while one exponentiates (the
-// special-function unit), the other loads, masks and stores.  A ninth warp's first thread issues all
-// tensor-core and TMA work: S = Q K^T two tiles ahead (8 instructions of K = 16, operands straight from
-// the swizzled TMA tiles: Q and K are K-major), O_g += P V as soon as a P is written (V is the MN-major
-// operand, the same swizzled tile as it arrived by TMA), stage refills once a tile's P V is complete.
+// special-function unit), the other loads, masks and stores.  A ninth warp's first thread issues the
+// tensor-core work: S = Q K^T two tiles ahead (8 instructions of K = 16, operands straight from the
+// swizzled TMA tiles: Q and K are K-major), O_g += P V as soon as a P is written (V is the MN-major
+// operand, the same swizzled tile as it arrived by TMA).  A tenth warp's first thread is the TMA
+// producer: it refills a stage's K as soon as the S that read it is complete and its V once its P V is.
 // A stream rescales its O in tensor memory only when a row's running maximum grows.  After the last
 // tile the two streams are combined like two splits, in registers.
 // =====================================================================================================
-#define UM_THREADS 288                               // two softmax warpgroups + the issuing warp
+#define UM_THREADS 320                               // two softmax warpgroups + the issuing warp + the TMA producer warp
 #define UM_ROWS_THREADS 128
 #define UM_SM_THREADS 256                            // softmax threads: row = tid & 127, stream = tid >> 7
 #define UM_P_BYTES (ATT_BM * ATT_BN * 2)             // 16 KiB: P tile, 128 rows x 64 keys bf16
@@ -441,16 +442,18 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const unsigned int sQ = smem_base + UM_STAGES * ATT_STAGE_BYTES;
     const unsigned int sP = sQ + ATT_Q_BYTES;
-    // barriers: K-full[UM_STAGES], V-full[UM_STAGES], S-ready[2], PV-done[2], partials-received, all-MMAs-done,
-    // P-written[2]; then the tensor-memory base.  S-ready, PV-done and P-written alternate with the tile's parity: a
-    // parity wait can only tell the current phase from the one before, and with two barriers the thread that waits
-    // for tile i is never more than one completion behind (the next completion on the same barrier is tile i + 2's).
-    const unsigned int bar0 = sP + 2 * UM_P_BYTES, bar_v = bar0 + UM_STAGES * 8;
-    const unsigned int bar_s = bar_v + UM_STAGES * 8, bar_pv = bar_s + 16, bar_r = bar_pv + 16, bar_done = bar_r + 8,
+    // barriers: K-full[UM_STAGES], V-full[UM_STAGES], K-free[UM_STAGES], V-free[UM_STAGES], S-ready[2],
+    // partials-received, all-MMAs-done, P-written[2]; then the tensor-memory base.  A parity wait can only tell the
+    // current phase from the one before, so every barrier is laid out such that its next completion depends on the
+    // thread that waits: a stage's barriers complete once per UM_STAGES tiles, S-ready and P-written alternate with
+    // the tile's parity.
+    const unsigned int bar0 = sP + 2 * UM_P_BYTES, bar_v = bar0 + UM_STAGES * 8, bar_ek = bar_v + UM_STAGES * 8,
+                       bar_ev = bar_ek + UM_STAGES * 8;
+    const unsigned int bar_s = bar_ev + UM_STAGES * 8, bar_r = bar_s + 16, bar_done = bar_r + 8,
                        bar_p = bar_done + 8, tslot = bar_p + 16;
     unsigned char* gQ = smem_gen + UM_STAGES * ATT_STAGE_BYTES;
     unsigned char* gP = gQ + ATT_Q_BYTES;
-    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + 2 * UM_P_BYTES + (2 * UM_STAGES + 8) * 8);
+    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + 2 * UM_P_BYTES + (4 * UM_STAGES + 6) * 8);
     float* s_mx = reinterpret_cast<float*>(gP + 2 * UM_P_BYTES + 1024);      // [2][128]: the streams' row maxima at the end
     float* s_lx = s_mx + 2 * ATT_BM;                                     // [2][128]: the streams' row sums
 
@@ -479,7 +482,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     };
     const int pre = min(np, UM_STAGES);
     if (tid == 0) {
-        for (int i = 0; i < 2 * UM_STAGES + 6; ++i) mbar_init(bar0 + i * 8, 1);
+        for (int i = 0; i < 4 * UM_STAGES + 4; ++i) mbar_init(bar0 + i * 8, 1);
         mbar_init(bar_p, UM_ROWS_THREADS);               // P of a tile is written: one arrival per thread of the stream
         mbar_init(bar_p + 8, UM_ROWS_THREADS);
         mbar_init_fence();
@@ -596,6 +599,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
             umma_ss_bf16(ts, dq0 + (qoffb >> 4), dk + (koffb >> 4), idesc_qk, ks > 0 ? 1u : 0u);
         }
         umma_commit(bar_s + (i & 1) * 8);
+        if (i + UM_STAGES < np) umma_commit(bar_ek + stage * 8);     // (the producer waits for it only then)
     };
     // O of stream i & 1 += P V of tile i (waits for V if it comes by TMA), then commit
     auto issue_pv = [&](int i) {
@@ -608,32 +612,48 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk)                       // 16 keys per instruction: two 8-key groups of V
             umma_ss_bf16(to, dp + (kk * 32 >> 4), dv + (kk * 2048 >> 4), idesc_pv, (i > 1 || kk > 0) ? 1u : 0u);
-        umma_commit(bar_pv + (i & 1) * 8);
+        umma_commit(bar_ev + stage * 8);
     };
     float mrun = -CUDART_INF_F, lrun = 0.f;
 
     // ---- KV tiles ------------------------------------------------------------------------------------------
-    if (tid == UM_SM_THREADS) {
-        // The issuing thread: S two tiles ahead of the softmax, O += P V as soon as a P is written; refills: K of
-        // tile i + 4 (S of tile i is long complete; waited for before S of tile i + 2 is committed to the same
-        // barrier) and V of tile i + 3 (once O += P V of tile i - 1 is complete).
-        if (ntiles > 0) issue_qk(0);
-        if (ntiles > 1) issue_qk(1);
+    // Both single-thread roles sit behind a branch on a warp-uniform value with the thread chosen by elect.sync in
+    // every round (all lanes run the loop): the compiler then keeps loop counters, addresses and descriptors uniform.
+    const int warp_u = __shfl_sync(HS_FULL_MASK, warp, 0);
+    if (warp_u == 8) {
+        // The issuing warp: S two tiles ahead of the softmax, O += P V as soon as a P is written.
+        if (elect_one()) {
+            if (ntiles > 0) issue_qk(0);
+            if (ntiles > 1) issue_qk(1);
+        }
+        __syncwarp();
 #pragma unroll 1
         for (int i = 0; i < ntiles; ++i) {
-            mbar_wait(bar_p + (i & 1) * 8, (unsigned int)(i >> 1) & 1u, p.err);   // P of tile i is written, its S is read
-            issue_pv(i);
-            if (i + UM_STAGES < np) {                        // S of tile i is complete (it was read): K's stage is free
-                mbar_wait(bar_s + (i & 1) * 8, (unsigned int)(i >> 1) & 1u, p.err);
-                issue_kv(i + UM_STAGES, false);
+            if (elect_one()) {
+                mbar_wait(bar_p + (i & 1) * 8, (unsigned int)(i >> 1) & 1u, p.err);   // P of tile i is written, its S is read
+                issue_pv(i);
+                if (i + 2 < ntiles) issue_qk(i + 2);
+                if (i == ntiles - 1) umma_commit(bar_done);      // every tensor-core operation of this CTA is complete
             }
-            if (i + 2 < ntiles) issue_qk(i + 2);
-            if (i >= 1 && i - 1 + UM_STAGES < np) {          // V's stage of tile i - 1 is free once its P V is done
-                mbar_wait(bar_pv + ((i - 1) & 1) * 8, (unsigned int)((i - 1) >> 1) & 1u, p.err);
-                issue_kv(i - 1 + UM_STAGES, true);
-            }
+            __syncwarp();
         }
-        if (ntiles > 0) umma_commit(bar_done);               // every tensor-core operation of this CTA is complete
+    } else if (warp_u == 9) {
+        // The TMA producer, in the order in which the tensor pipe frees the stages: K of tile t (its stage was
+        // read by S of tile t - UM_STAGES), then V of tile t - 1.
+#pragma unroll 1
+        for (int t = UM_STAGES; t <= np; ++t) {
+            if (elect_one()) {
+                if (t < np) {
+                    mbar_wait(bar_ek + (t % UM_STAGES) * 8, (unsigned int)(t / UM_STAGES - 1) & 1u, p.err);
+                    issue_kv(t, false);
+                }
+                if (t - 1 >= UM_STAGES) {
+                    mbar_wait(bar_ev + ((t - 1) % UM_STAGES) * 8, (unsigned int)((t - 1) / UM_STAGES - 1) & 1u, p.err);
+                    issue_kv(t - 1, true);
+                }
+            }
+            __syncwarp();
+        }
     }
     // Stream `half`: tiles half, half + 2, ...  What a stream touches at tile i (its S and P buffers, its O) was
     // last used by the tensor cores for tile i - 2, and S of tile i was committed after O += P V of tile i - 2 was
@@ -689,11 +709,10 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         }
         lrun = fmaf(lrun, corr, lsa + lsb);
         // A tree tile is gathered into the stage of tile i - 1 once that tile's O += P V is complete (a prefix tile
-        // is requested by the issuing thread).  P of tile i + 1 is not written before this stream's P of tile i is,
-        // so the barrier of tile i - 1's parity cannot be a phase ahead: the parity wait is unambiguous.
+        // is requested by the producer thread).  The barrier's next completion is tile nx's own P V.
         const int nx = i - 1 + UM_STAGES;
         if (i >= 1 && nx < ntiles && nx >= np) {
-            mbar_wait(bar_pv + ((i - 1) & 1) * 8, (unsigned int)((i - 1) >> 1) & 1u, p.err);
+            mbar_wait(bar_ev + ((i - 1) % UM_STAGES) * 8, (unsigned int)((i - 1) / UM_STAGES) & 1u, p.err);
             gather_tree(nx, row, UM_ROWS_THREADS, 0);
             gather_tree(nx, row, UM_ROWS_THREADS, 4);
         }
@@ -718,7 +737,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         mbar_arrive(bar_p + half * 8);
     }
     if (ntiles > 0 && warp < 8) mbar_wait(bar_done, 0u, p.err);
-    __syncwarp();                                        // the issuing warp reconverges (warp-aligned barriers follow)
+    __syncwarp();                                        // the issuing and producer warps reconverge (warp-aligned barriers follow)
     tc_fence_after_sync();
     // the two streams of a row are combined like two splits: weights w0, w1 on the streams' O, one (max, sum)
     if (warp < 8) { s_mx[half * ATT_BM + row] = mrun; s_lx[half * ATT_BM + row] = lrun; }
