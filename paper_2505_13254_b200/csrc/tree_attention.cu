@@ -443,17 +443,17 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     const unsigned int sQ = smem_base + UM_STAGES * ATT_STAGE_BYTES;
     const unsigned int sP = sQ + ATT_Q_BYTES;
     // barriers: K-full[UM_STAGES], V-full[UM_STAGES], K-free[UM_STAGES], V-free[UM_STAGES], S-ready[2],
-    // partials-received, all-MMAs-done, P-written[2]; then the tensor-memory base.  A parity wait can only tell the
+    // partials-received, all-MMAs-done, P-written[2], S-read[2]; then the tensor-memory base.  A parity wait can only tell the
     // current phase from the one before, so every barrier is laid out such that its next completion depends on the
     // thread that waits: a stage's barriers complete once per UM_STAGES tiles, S-ready and P-written alternate with
     // the tile's parity.
     const unsigned int bar0 = sP + 2 * UM_P_BYTES, bar_v = bar0 + UM_STAGES * 8, bar_ek = bar_v + UM_STAGES * 8,
                        bar_ev = bar_ek + UM_STAGES * 8;
     const unsigned int bar_s = bar_ev + UM_STAGES * 8, bar_r = bar_s + 16, bar_done = bar_r + 8,
-                       bar_p = bar_done + 8, tslot = bar_p + 16;
+                       bar_p = bar_done + 8, bar_sr = bar_p + 16, tslot = bar_sr + 16;
     unsigned char* gQ = smem_gen + UM_STAGES * ATT_STAGE_BYTES;
     unsigned char* gP = gQ + ATT_Q_BYTES;
-    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + 2 * UM_P_BYTES + (4 * UM_STAGES + 6) * 8);
+    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + 2 * UM_P_BYTES + (4 * UM_STAGES + 8) * 8);
     float* s_mx = reinterpret_cast<float*>(gP + 2 * UM_P_BYTES + 1024);      // [2][128]: the streams' row maxima at the end
     float* s_lx = s_mx + 2 * ATT_BM;                                     // [2][128]: the streams' row sums
 
@@ -485,6 +485,8 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         for (int i = 0; i < 4 * UM_STAGES + 4; ++i) mbar_init(bar0 + i * 8, 1);
         mbar_init(bar_p, UM_ROWS_THREADS);               // P of a tile is written: one arrival per thread of the stream
         mbar_init(bar_p + 8, UM_ROWS_THREADS);
+        mbar_init(bar_sr, UM_ROWS_THREADS);              // S of a tile is in registers: its buffer may take the next S
+        mbar_init(bar_sr + 8, UM_ROWS_THREADS);
         mbar_init_fence();
         for (int i = 0; i < pre; ++i) { issue_kv(i, false); issue_kv(i, true); }
     }
@@ -518,9 +520,9 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     const int nt_tree = (split == p.nsplit - 1) ? (nk + ATT_BN - 1) / ATT_BN : 0;
     const int ntiles = np + nt_tree;
 
-    // tree keys/values: gathered rows, 16-byte loads (four of a thread's loads in flight together), swizzled
-    // stores; 2 x 1024 chunks by nthr threads (thread t of them), chunks t + (it0 .. it0 + 3) * nthr
-    auto gather_tree = [&](int i, int t, int nthr, int it0) {
+    // tree keys and/or values of tile i: gathered rows, 16-byte loads (four of a thread's loads per matrix in flight
+    // together), swizzled stores; 1024 chunks per matrix by nthr threads (thread t of them), chunks t + (it0 .. it0 + 3) * nthr
+    auto gather_tree = [&](int i, int t, int nthr, int it0, bool do_k, bool do_v) {
         unsigned char* gK = smem_gen + (i % UM_STAGES) * ATT_STAGE_BYTES;
         unsigned char* gV = gK + ATT_TILE_BYTES;
         const int j0 = (i - np) * ATT_BN;
@@ -538,15 +540,15 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
             vvv[it] = make_uint4(0, 0, 0, 0);
             if (trow[it] >= 0) {
                 const size_t off = ((size_t)trow[it] * p.hkv + h) * HS_HEAD_DIM + (t & 15) * 8;
-                kvv[it] = __ldg(reinterpret_cast<const uint4*>(p.k_tree + off));
-                vvv[it] = __ldg(reinterpret_cast<const uint4*>(p.v_tree + off));
+                if (do_k) kvv[it] = __ldg(reinterpret_cast<const uint4*>(p.k_tree + off));
+                if (do_v) vvv[it] = __ldg(reinterpret_cast<const uint4*>(p.v_tree + off));
             }
         }
 #pragma unroll
         for (int it = 0; it < 4; ++it) {
             const int c = t + (it0 + it) * nthr;
-            *reinterpret_cast<uint4*>(gK + tile_off(c >> 4, c & 15)) = kvv[it];
-            *reinterpret_cast<uint4*>(gV + tile_off(c >> 4, c & 15)) = vvv[it];
+            if (do_k) *reinterpret_cast<uint4*>(gK + tile_off(c >> 4, c & 15)) = kvv[it];
+            if (do_v) *reinterpret_cast<uint4*>(gV + tile_off(c >> 4, c & 15)) = vvv[it];
         }
     };
 
@@ -574,7 +576,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         }
     }
     if (warp < 8)
-        for (int i = np; i < min(ntiles, UM_STAGES); ++i) gather_tree(i, tid, UM_SM_THREADS, 0);  // tree tiles that open the pipeline
+        for (int i = np; i < min(ntiles, UM_STAGES); ++i) gather_tree(i, tid, UM_SM_THREADS, 0, true, true);  // tree tiles that open the pipeline
     fence_proxy_async_smem();                        // generic stores -> visible to the tensor cores
     __syncthreads();
 
@@ -621,43 +623,59 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     // every round (all lanes run the loop): the compiler then keeps loop counters, addresses and descriptors uniform.
     const int warp_u = __shfl_sync(HS_FULL_MASK, warp, 0);
     if (warp_u == 8) {
-        // The issuing warp: S two tiles ahead of the softmax, O += P V as soon as a P is written.
+        // The issuing warp.  S of tile i + 2 is issued as soon as the stream has S of tile i in registers, so a
+        // stream never waits for its next S; O += P V of tile i as soon as its P is written.  Per stream the events
+        // come as "P of tile i written, S of tile i + 2 read", and the loop takes them in that order.
         if (elect_one()) {
             if (ntiles > 0) issue_qk(0);
             if (ntiles > 1) issue_qk(1);
+            for (int i = 0; i < 2 && i + 2 < ntiles; ++i) {
+                mbar_wait(bar_sr + i * 8, 0u, p.err);
+                issue_qk(i + 2);
+            }
         }
         __syncwarp();
 #pragma unroll 1
         for (int i = 0; i < ntiles; ++i) {
             if (elect_one()) {
-                mbar_wait(bar_p + (i & 1) * 8, (unsigned int)(i >> 1) & 1u, p.err);   // P of tile i is written, its S is read
+                mbar_wait(bar_p + (i & 1) * 8, (unsigned int)(i >> 1) & 1u, p.err);   // P of tile i is written
                 issue_pv(i);
-                if (i + 2 < ntiles) issue_qk(i + 2);
+                if (i + 4 < ntiles) {
+                    mbar_wait(bar_sr + (i & 1) * 8, (unsigned int)((i + 2) >> 1) & 1u, p.err);   // S of tile i + 2 is read
+                    issue_qk(i + 4);
+                }
                 if (i == ntiles - 1) umma_commit(bar_done);      // every tensor-core operation of this CTA is complete
             }
             __syncwarp();
         }
     } else if (warp_u == 9) {
-        // The TMA producer, in the order in which the tensor pipe frees the stages: K of tile t (its stage was
-        // read by S of tile t - UM_STAGES), then V of tile t - 1.
+        // The TMA producer, in the order in which the tensor pipe frees the stage halves: S runs four tiles ahead
+        // of O += P V, so after the first K refills it is V of tile i + 4 (after P V of tile i), then K of tile i + 8
+        // (after S of tile i + 4).
 #pragma unroll 1
-        for (int t = UM_STAGES; t <= np; ++t) {
+        for (int t = UM_STAGES; t < min(np, 2 * UM_STAGES); ++t) {
             if (elect_one()) {
-                if (t < np) {
-                    mbar_wait(bar_ek + (t % UM_STAGES) * 8, (unsigned int)(t / UM_STAGES - 1) & 1u, p.err);
-                    issue_kv(t, false);
-                }
-                if (t - 1 >= UM_STAGES) {
-                    mbar_wait(bar_ev + ((t - 1) % UM_STAGES) * 8, (unsigned int)((t - 1) / UM_STAGES - 1) & 1u, p.err);
-                    issue_kv(t - 1, true);
+                mbar_wait(bar_ek + (t % UM_STAGES) * 8, 0u, p.err);
+                issue_kv(t, false);
+            }
+            __syncwarp();
+        }
+#pragma unroll 1
+        for (int i = 0; i + UM_STAGES < np; ++i) {
+            if (elect_one()) {
+                mbar_wait(bar_ev + (i % UM_STAGES) * 8, (unsigned int)(i / UM_STAGES) & 1u, p.err);
+                issue_kv(i + UM_STAGES, true);
+                if (i + 2 * UM_STAGES < np) {
+                    mbar_wait(bar_ek + (i % UM_STAGES) * 8, (unsigned int)(i / UM_STAGES + 1) & 1u, p.err);
+                    issue_kv(i + 2 * UM_STAGES, false);
                 }
             }
             __syncwarp();
         }
     }
-    // Stream `half`: tiles half, half + 2, ...  What a stream touches at tile i (its S and P buffers, its O) was
-    // last used by the tensor cores for tile i - 2, and S of tile i was committed after O += P V of tile i - 2 was
-    // issued: once S is there, nothing else has to be waited for.
+    // Stream `half`: tiles half, half + 2, ...  As soon as S of tile i is in registers its buffer is handed back.  The
+    // stream's P buffer and O were last used by O += P V of tile i - 2, which is waited for before they are touched
+    // (its barrier's next completion is tile i + 2's, which needs this stream's P of tile i + 2).
 #pragma unroll 1
     for (int i = half; i < ntiles && warp < 8; i += 2) {
         mbar_wait(bar_s + half * 8, (unsigned int)(i >> 1) & 1u, p.err);         // S of tile i is complete
@@ -666,6 +684,8 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         tmem_ld32(tS + half * ATT_BN + lane_off, sr);
         tmem_ld32(tS + half * ATT_BN + 32 + lane_off, sr + 32);
         tmem_wait_ld();
+        tc_fence_before_sync();
+        mbar_arrive(bar_sr + half * 8);
 
         const bool is_tree = i >= np;
         const int col0 = is_tree ? (i - np) * ATT_BN : (t0 + i) * ATT_BN;
@@ -708,13 +728,20 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
             pk[c8].z = pack_bf16(pv[4], pv[5]); pk[c8].w = pack_bf16(pv[6], pv[7]);
         }
         lrun = fmaf(lrun, corr, lsa + lsb);
-        // A tree tile is gathered into the stage of tile i - 1 once that tile's O += P V is complete (a prefix tile
-        // is requested by the producer thread).  The barrier's next completion is tile nx's own P V.
-        const int nx = i - 1 + UM_STAGES;
-        if (i >= 1 && nx < ntiles && nx >= np) {
-            mbar_wait(bar_ev + ((i - 1) % UM_STAGES) * 8, (unsigned int)((i - 1) / UM_STAGES) & 1u, p.err);
-            gather_tree(nx, row, UM_ROWS_THREADS, 0);
-            gather_tree(nx, row, UM_ROWS_THREADS, 4);
+        // Tree tiles are gathered by the stream two and four tiles ahead of their use, where the stage half is free
+        // and this tile's P-written arrival publishes the stores before the issuing thread needs them: K of tile
+        // i + 4 (its stage's K was read by S of tile i, complete), V of tile i + 2 (after O += P V of tile i - 2).
+        if (i + UM_STAGES < ntiles && i + UM_STAGES >= np) {
+            gather_tree(i + UM_STAGES, row, UM_ROWS_THREADS, 0, true, false);
+            gather_tree(i + UM_STAGES, row, UM_ROWS_THREADS, 4, true, false);
+        }
+        if (i >= 2) {
+            mbar_wait(bar_ev + ((i - 2) % UM_STAGES) * 8, (unsigned int)((i - 2) / UM_STAGES) & 1u, p.err);
+            tc_fence_after_sync();
+            if (i + 2 < ntiles && i + 2 >= np) {
+                gather_tree(i + 2, row, UM_ROWS_THREADS, 0, false, true);
+                gather_tree(i + 2, row, UM_ROWS_THREADS, 4, false, true);
+            }
         }
         // rescale this stream's O (the load/store are warp-wide: a warp rescales if any of its rows needs it)
         if (i >= 2 && __any_sync(HS_FULL_MASK, corr != 1.f)) {
