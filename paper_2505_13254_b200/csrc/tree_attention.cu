@@ -412,15 +412,15 @@ tree_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, co
 // rows: warpgroup g takes the KV tiles i = g, g + 2, ... and keeps its own S buffer, P buffer, running
 // (max, sum) and O accumulator; thread t of a warpgroup owns query row t (= tensor-memory lane t), so the
 // softmax needs no shuffles and the two streams never wait for one another: while one exponentiates (the
-// special-function unit), the other loads, masks and stores.  A ninth warp's first thread issues the
-// tensor-core work: S = Q K^T two tiles ahead (8 instructions of K = 16, operands straight from the
-// swizzled TMA tiles: Q and K are K-major), O_g += P V as soon as a P is written (V is the MN-major
-// operand, the same swizzled tile as it arrived by TMA).  A tenth warp's first thread is the TMA
-// producer: it refills a stage's K as soon as the S that read it is complete and its V once its P V is.
+// special-function unit), the other loads, masks and stores.  Three more warps give one elected thread each: the S issuer
+// (S = Q K^T of tile i + 2 as soon as S of tile i is in registers; 8 instructions of K = 16, operands
+// straight from the swizzled TMA tiles: Q and K are K-major), the P V issuer (O_g += P V as soon as a P
+// is written; V is the MN-major operand, the same swizzled tile as it arrived by TMA) and the TMA
+// producer (a stage's K is refilled as soon as the S that read it is complete, its V once its P V is).
 // A stream rescales its O in tensor memory only when a row's running maximum grows.  After the last
 // tile the two streams are combined like two splits, in registers.
 // =====================================================================================================
-#define UM_THREADS 320                               // two softmax warpgroups + the issuing warp + the TMA producer warp
+#define UM_THREADS 352                               // two softmax warpgroups + P V issuer, TMA producer, S issuer warps
 #define UM_ROWS_THREADS 128
 #define UM_SM_THREADS 256                            // softmax threads: row = tid & 127, stream = tid >> 7
 #define UM_P_BYTES (ATT_BM * ATT_BN * 2)             // 16 KiB: P tile, 128 rows x 64 keys bf16
@@ -623,28 +623,32 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     // every round (all lanes run the loop): the compiler then keeps loop counters, addresses and descriptors uniform.
     const int warp_u = __shfl_sync(HS_FULL_MASK, warp, 0);
     if (warp_u == 8) {
-        // The issuing warp.  S of tile i + 2 is issued as soon as the stream has S of tile i in registers, so a
-        // stream never waits for its next S; O += P V of tile i as soon as its P is written.  Per stream the events
-        // come as "P of tile i written, S of tile i + 2 read", and the loop takes them in that order.
-        if (elect_one()) {
-            if (ntiles > 0) issue_qk(0);
-            if (ntiles > 1) issue_qk(1);
-            for (int i = 0; i < 2 && i + 2 < ntiles; ++i) {
-                mbar_wait(bar_sr + i * 8, 0u, p.err);
-                issue_qk(i + 2);
-            }
-        }
-        __syncwarp();
+        // The P V issuer: O += P V of tile i as soon as its P is written.  It is short work on the streams' critical
+        // path (a stream may not write P of tile i + 2 before it is complete), so it has a thread of its own that is
+        // never held up behind the issue of an S.
 #pragma unroll 1
         for (int i = 0; i < ntiles; ++i) {
             if (elect_one()) {
                 mbar_wait(bar_p + (i & 1) * 8, (unsigned int)(i >> 1) & 1u, p.err);   // P of tile i is written
                 issue_pv(i);
-                if (i + 4 < ntiles) {
-                    mbar_wait(bar_sr + (i & 1) * 8, (unsigned int)((i + 2) >> 1) & 1u, p.err);   // S of tile i + 2 is read
-                    issue_qk(i + 4);
-                }
-                if (i == ntiles - 1) umma_commit(bar_done);      // every tensor-core operation of this CTA is complete
+                // every S was read before the last P was written: all tensor-core work of this CTA is complete
+                if (i == ntiles - 1) umma_commit(bar_done);
+            }
+            __syncwarp();
+        }
+    } else if (warp_u == 10) {
+        // The S issuer: S of tile i + 2 as soon as the stream has S of tile i in registers, so a stream never waits
+        // for its next S.
+        if (elect_one()) {
+            if (ntiles > 0) issue_qk(0);
+            if (ntiles > 1) issue_qk(1);
+        }
+        __syncwarp();
+#pragma unroll 1
+        for (int i = 0; i + 2 < ntiles; ++i) {
+            if (elect_one()) {
+                mbar_wait(bar_sr + (i & 1) * 8, (unsigned int)(i >> 1) & 1u, p.err);      // S of tile i is read
+                issue_qk(i + 2);
             }
             __syncwarp();
         }
