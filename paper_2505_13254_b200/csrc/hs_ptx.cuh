@@ -135,6 +135,16 @@ __device__ __forceinline__ void umma_ss_bf16(unsigned int d_tmem, unsigned long 
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
         : "memory");
 }
+// D[tmem] (+)= A[tmem] * B[smem]: A's 128 rows are the tensor-memory lanes, its K = 16 bf16 elements fill 8
+// consecutive 32-bit columns (two elements per column, the lower index in the low half).
+__device__ __forceinline__ void umma_ts_bf16(unsigned int d_tmem, unsigned int a_tmem, unsigned long long b_desc,
+                                             unsigned int idesc, unsigned int accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %6, %7, %8}, p;\n\t}\n"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
+        : "memory");
+}
 // mbarrier arrives once all tensor-core operations issued so far by this thread have completed
 __device__ __forceinline__ void umma_commit(unsigned int bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");

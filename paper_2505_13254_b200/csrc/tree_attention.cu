@@ -424,7 +424,7 @@ tree_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, co
 #define UM_ROWS_THREADS 128
 #define UM_SM_THREADS 256                            // softmax threads: row = tid & 127, stream = tid >> 7
 #define UM_P_BYTES (ATT_BM * ATT_BN * 2)             // 16 KiB: P tile, 128 rows x 64 keys bf16
-#define UM_TMEM_COLS 512                             // S of stream g: columns 64 g ..; O of stream g: columns 128 + 128 g ..
+#define UM_TMEM_COLS 512                             // S of stream g: columns 64 g ..; O: 128 + 128 g ..; P (bf16 pairs): 384 + 32 g ..
 #define UM_STAGES 4
 #define UM_RECV_BYTES (76 * 1024)                    // after the tile loop: partials pushed by the splits of the cluster
 #define UM_SMEM_BYTES (UM_STAGES * ATT_STAGE_BYTES + ATT_Q_BYTES + 2 * UM_P_BYTES + 4096 + 1024)
@@ -502,7 +502,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     const unsigned int tmem_base = *tslot_gen;
     const unsigned int lane_off = (unsigned int)((warp & 3) * 32) << 16;   // a warp reaches lanes 32 * (warp % 4) ...
     const int row = tid & (ATT_BM - 1), half = (tid >> 7) & 1;               // the thread's query row and stream
-    const unsigned int tS = tmem_base, tO = tmem_base + 128;                 // (+ 64 / + 128 columns for stream 1)
+    const unsigned int tS = tmem_base, tO = tmem_base + 128, tP = tmem_base + 384;   // (+ 64 / + 128 / + 32 columns for stream 1)
 
     const int nk = (p.status[b] == 0) ? p.n_keep[b] : 0;
     const int M = nk * p.G;
@@ -585,8 +585,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     // Operand descriptors: the start-address field (16-byte units, low 14 bits) is the only part that varies, and no
     // shared-memory address reaches 2^18, so an offset is added to a descriptor built once.
     const unsigned long long dq0 = umma_desc_sw128(sQ, 16, 1024), dk0 = umma_desc_sw128(smem_base, 16, 1024);
-    const unsigned long long dp0 = umma_desc_sw128(sP, 16, 1024),
-                             dv0 = umma_desc_sw128(smem_base + ATT_TILE_BYTES, ATT_TILE_BYTES / 2, 1024);
+    const unsigned long long dv0 = umma_desc_sw128(smem_base + ATT_TILE_BYTES, ATT_TILE_BYTES / 2, 1024);
     // the issuing thread: S = Q K^T of tile i into S buffer i & 1 (waits for K if it comes by TMA), then commit
     auto issue_qk = [&](int i) {
         const int stage = i % UM_STAGES;
@@ -609,11 +608,11 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         if (i < np) mbar_wait(bar_v + stage * 8, (unsigned int)(i / UM_STAGES) & 1u, p.err);
         tc_fence_after_sync();
         const unsigned long long dv = dv0 + (unsigned long long)(stage * (ATT_STAGE_BYTES >> 4));
-        const unsigned long long dp = dp0 + (unsigned long long)((i & 1) * (UM_P_BYTES >> 4));
+        const unsigned int tp = tP + (i & 1) * (ATT_BN / 2);
         const unsigned int to = tO + (i & 1) * HS_HEAD_DIM;
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk)                       // 16 keys per instruction: two 8-key groups of V
-            umma_ss_bf16(to, dp + (kk * 32 >> 4), dv + (kk * 2048 >> 4), idesc_pv, (i > 1 || kk > 0) ? 1u : 0u);
+            umma_ts_bf16(to, tp + kk * 8, dv + (kk * 2048 >> 4), idesc_pv, (i > 1 || kk > 0) ? 1u : 0u);
         umma_commit(bar_ev + stage * 8);
     };
     float mrun = -CUDART_INF_F, lrun = 0.f;
@@ -760,10 +759,10 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
             }
             tmem_wait_st();
         }
-#pragma unroll
-        for (int c8 = 0; c8 < 8; ++c8)
-            *reinterpret_cast<uint4*>(gP + half * UM_P_BYTES + row * 128 + ((c8 ^ (row & 7)) << 4)) = pk[c8];
-        fence_proxy_async_smem();                            // P (and gathered tree tiles) -> tensor cores
+        // P stays in tensor memory (the A operand of O += P V): this row's 64 bf16 values are 32 columns of its lane
+        tmem_st32(tP + half * (ATT_BN / 2) + lane_off, reinterpret_cast<unsigned int*>(pk));
+        tmem_wait_st();
+        if (i + UM_STAGES >= np) fence_proxy_async_smem();   // gathered tree tiles (generic stores) -> tensor cores
         tc_fence_before_sync();
         mbar_arrive(bar_p + half * 8);
     }
