@@ -35,6 +35,7 @@ def run_and_check(ctx, cfg, policy, seed, attention="full", **kw):
         snap = [t.clone() for t in (st.quant.h_full, st.quant.phi, st.pruned.anc_mask, st.accept.path_nodes)]
         if attention != "none":
             snap.append(st.attn_out.clone())
+        assert hb.hs_device_error(ctx) == 0     # no device-side wait gave up
         if rep == 1:
             assert all(torch.equal(a, b) for a, b in zip(snap, first))
         first = snap
