@@ -424,7 +424,7 @@ tree_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, co
 #define UM_ROWS_THREADS 128
 #define UM_SM_THREADS 256                            // softmax threads: row = tid & 127, stream = tid >> 7
 #define UM_P_BYTES (ATT_BM * ATT_BN * 2)             // 16 KiB: P tile, 128 rows x 64 keys bf16
-#define UM_TMEM_COLS 512                             // S of stream g: columns 64 g ..; O: 128 + 128 g ..; P (bf16 pairs, two buffers): 384 + 64 g ..
+#define UM_TMEM_COLS 512                             // S of stream g: columns 64 g ..; O: 128 + 128 g ..; P (bf16 pairs): 384 + 32 g ..
 #define UM_STAGES 4
 #define UM_RECV_BYTES (76 * 1024)                    // after the tile loop: partials pushed by the splits of the cluster
 #define UM_SMEM_BYTES (UM_STAGES * ATT_STAGE_BYTES + ATT_Q_BYTES + 2 * UM_P_BYTES + 4096 + 1024)
@@ -443,18 +443,17 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     const unsigned int sQ = smem_base + UM_STAGES * ATT_STAGE_BYTES;
     const unsigned int sP = sQ + ATT_Q_BYTES;
     // barriers: K-full[UM_STAGES], V-full[UM_STAGES], K-free[UM_STAGES], V-free[UM_STAGES], S-ready[2],
-    // partials-received, all-MMAs-done, P-written[4], S-read[2]; then the tensor-memory base.  A parity wait can only tell the
+    // partials-received, all-MMAs-done, P-written[2], S-read[2]; then the tensor-memory base.  A parity wait can only tell the
     // current phase from the one before, so every barrier is laid out such that its next completion depends on the
-    // thread that waits: a stage's barriers complete once per UM_STAGES tiles, S-ready and S-read alternate with
-    // the tile's parity, P-written goes round over four barriers (P is double-buffered per stream, so a stream can be
-    // two of its tiles ahead of the P V issuer).
+    // thread that waits: a stage's barriers complete once per UM_STAGES tiles, S-ready and P-written alternate with
+    // the tile's parity.
     const unsigned int bar0 = sP + 2 * UM_P_BYTES, bar_v = bar0 + UM_STAGES * 8, bar_ek = bar_v + UM_STAGES * 8,
                        bar_ev = bar_ek + UM_STAGES * 8;
     const unsigned int bar_s = bar_ev + UM_STAGES * 8, bar_r = bar_s + 16, bar_done = bar_r + 8,
-                       bar_p = bar_done + 8, bar_sr = bar_p + 32, tslot = bar_sr + 16;
+                       bar_p = bar_done + 8, bar_sr = bar_p + 16, tslot = bar_sr + 16;
     unsigned char* gQ = smem_gen + UM_STAGES * ATT_STAGE_BYTES;
     unsigned char* gP = gQ + ATT_Q_BYTES;
-    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + 2 * UM_P_BYTES + (4 * UM_STAGES + 10) * 8);
+    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + 2 * UM_P_BYTES + (4 * UM_STAGES + 8) * 8);
     float* s_mx = reinterpret_cast<float*>(gP + 2 * UM_P_BYTES + 1024);      // [2][128]: the streams' row maxima at the end
     float* s_lx = s_mx + 2 * ATT_BM;                                     // [2][128]: the streams' row sums
 
@@ -484,7 +483,8 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     const int pre = min(np, UM_STAGES);
     if (tid == 0) {
         for (int i = 0; i < 4 * UM_STAGES + 4; ++i) mbar_init(bar0 + i * 8, 1);
-        for (int i = 0; i < 4; ++i) mbar_init(bar_p + i * 8, UM_ROWS_THREADS);   // P of a tile is written: one arrival per thread of the stream
+        mbar_init(bar_p, UM_ROWS_THREADS);               // P of a tile is written: one arrival per thread of the stream
+        mbar_init(bar_p + 8, UM_ROWS_THREADS);
         mbar_init(bar_sr, UM_ROWS_THREADS);              // S of a tile is in registers: its buffer may take the next S
         mbar_init(bar_sr + 8, UM_ROWS_THREADS);
         mbar_init_fence();
@@ -502,7 +502,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     const unsigned int tmem_base = *tslot_gen;
     const unsigned int lane_off = (unsigned int)((warp & 3) * 32) << 16;   // a warp reaches lanes 32 * (warp % 4) ...
     const int row = tid & (ATT_BM - 1), half = (tid >> 7) & 1;               // the thread's query row and stream
-    const unsigned int tS = tmem_base, tO = tmem_base + 128, tP = tmem_base + 384;   // (+ 64 / + 128 / + 64 columns for stream 1)
+    const unsigned int tS = tmem_base, tO = tmem_base + 128, tP = tmem_base + 384;   // (+ 64 / + 128 / + 32 columns for stream 1)
 
     const int nk = (p.status[b] == 0) ? p.n_keep[b] : 0;
     const int M = nk * p.G;
@@ -608,7 +608,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         if (i < np) mbar_wait(bar_v + stage * 8, (unsigned int)(i / UM_STAGES) & 1u, p.err);
         tc_fence_after_sync();
         const unsigned long long dv = dv0 + (unsigned long long)(stage * (ATT_STAGE_BYTES >> 4));
-        const unsigned int tp = tP + (i & 1) * ATT_BN + ((i >> 1) & 1) * (ATT_BN / 2);
+        const unsigned int tp = tP + (i & 1) * (ATT_BN / 2);
         const unsigned int to = tO + (i & 1) * HS_HEAD_DIM;
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk)                       // 16 keys per instruction: two 8-key groups of V
@@ -628,7 +628,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
 #pragma unroll 1
         for (int i = 0; i < ntiles; ++i) {
             if (elect_one()) {
-                mbar_wait(bar_p + (i & 3) * 8, (unsigned int)(i >> 2) & 1u, p.err);   // P of tile i is written
+                mbar_wait(bar_p + (i & 1) * 8, (unsigned int)(i >> 1) & 1u, p.err);   // P of tile i is written
                 issue_pv(i);
                 // every S was read before the last P was written: all tensor-core work of this CTA is complete
                 if (i == ntiles - 1) umma_commit(bar_done);
@@ -708,29 +708,52 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
             }
         }
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-            mxa = fmaxf(mxa, __uint_as_float(sr[c]));
-            mxb = fmaxf(mxb, __uint_as_float(sr[32 + c]));
+        for (int c = 0; c < 32; c += 2) {                    // three-input maxima: half the instructions
+            mxa = max3(mxa, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
+            mxb = max3(mxb, __uint_as_float(sr[32 + c]), __uint_as_float(sr[33 + c]));
         }
         const float mx = fmaxf(mxa, mxb) * p.scale_log2;
         const float mnew = fmaxf(mrun, mx);
         const float muse = (mnew == -CUDART_INF_F) ? 0.f : mnew;
         const float corr = ex2_approx(mrun - muse);          // 1 when the maximum did not grow, 0 at the stream's first tile
         mrun = mnew;
-        lrun *= corr;
-        // What the stream touches besides its S: its O (only if a row maximum grew: rescale) and the stage of tile
-        // i - 2 (only if tile i + 2 is a tree tile: its V is gathered there) need O += P V of tile i - 2 complete;
-        // P is double-buffered, and the buffer of tile i was last read by O += P V of tile i - 4.  Each of these
-        // barriers completes next for a tile whose P this stream has not written yet.
-        const bool rescale = i >= 2 && __any_sync(HS_FULL_MASK, corr != 1.f);
-        const bool gather_v = i >= 2 && i + 2 < ntiles && i + 2 >= np;
-        if (rescale || gather_v) {
-            mbar_wait(bar_ev + ((i - 2) % UM_STAGES) * 8, (unsigned int)((i - 2) / UM_STAGES) & 1u, p.err);
-        } else if (i >= UM_STAGES) {
-            mbar_wait(bar_ev + (i % UM_STAGES) * 8, (unsigned int)(i / UM_STAGES - 1) & 1u, p.err);
+        // the row's P of this tile, in registers first
+        // (the exponent's multiply-add and the row sum run as packed fp32 pairs: half the instructions)
+        const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(-muse, -muse);
+        float2 ls0 = make_float2(0.f, 0.f), ls1 = make_float2(0.f, 0.f);
+        uint4 pk[8];
+#pragma unroll
+        for (int c8 = 0; c8 < 8; ++c8) {
+            float2 pv[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 x = fma2_ftz(make_float2(__uint_as_float(sr[c8 * 8 + 2 * e]), __uint_as_float(sr[c8 * 8 + 2 * e + 1])), sc2, nm2);
+                pv[e] = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+            }
+            ls0 = add2_ftz(ls0, add2_ftz(pv[0], pv[1]));
+            ls1 = add2_ftz(ls1, add2_ftz(pv[2], pv[3]));
+            pk[c8].x = pack_bf16(pv[0].x, pv[0].y); pk[c8].y = pack_bf16(pv[1].x, pv[1].y);
+            pk[c8].z = pack_bf16(pv[2].x, pv[2].y); pk[c8].w = pack_bf16(pv[3].x, pv[3].y);
         }
-        tc_fence_after_sync();
-        if (rescale) {       // (the load/store are warp-wide: a warp rescales if any of its rows needs it)
+        const float2 ls = add2_ftz(ls0, ls1);
+        lrun = fmaf(lrun, corr, ls.x + ls.y);
+        // Tree tiles are gathered by the stream two and four tiles ahead of their use, where the stage half is free
+        // and this tile's P-written arrival publishes the stores before the issuing thread needs them: K of tile
+        // i + 4 (its stage's K was read by S of tile i, complete), V of tile i + 2 (after O += P V of tile i - 2).
+        if (i + UM_STAGES < ntiles && i + UM_STAGES >= np) {
+            gather_tree(i + UM_STAGES, row, UM_ROWS_THREADS, 0, true, false);
+            gather_tree(i + UM_STAGES, row, UM_ROWS_THREADS, 4, true, false);
+        }
+        if (i >= 2) {
+            mbar_wait(bar_ev + ((i - 2) % UM_STAGES) * 8, (unsigned int)((i - 2) / UM_STAGES) & 1u, p.err);
+            tc_fence_after_sync();
+            if (i + 2 < ntiles && i + 2 >= np) {
+                gather_tree(i + 2, row, UM_ROWS_THREADS, 0, false, true);
+                gather_tree(i + 2, row, UM_ROWS_THREADS, 4, false, true);
+            }
+        }
+        // rescale this stream's O (the load/store are warp-wide: a warp rescales if any of its rows needs it)
+        if (i >= 2 && __any_sync(HS_FULL_MASK, corr != 1.f)) {
 #pragma unroll 1
             for (int ch = 0; ch < 4; ++ch) {
                 unsigned int ov[32];
@@ -740,45 +763,14 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
                 for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * corr);
                 tmem_st32(tO + half * HS_HEAD_DIM + lane_off + ch * 32, ov);
             }
+            tmem_wait_st();
         }
-        // The row's P of this tile stays in tensor memory (the A operand of O += P V): 64 bf16 values = 32 columns of
-        // the row's lane, stored in two halves so that the first store is in flight under the second half's exponentials.
-        const unsigned int tp = tP + half * ATT_BN + ((i >> 1) & 1) * (ATT_BN / 2) + lane_off;
-        float lsa = 0.f, lsb = 0.f;
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-            unsigned int pk[16];
-#pragma unroll
-            for (int c8 = 0; c8 < 4; ++c8) {
-                float pv[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e)
-                    pv[e] = ex2_approx(fmaf(__uint_as_float(sr[hh * 32 + c8 * 8 + e]), p.scale_log2, -muse));
-                lsa += (pv[0] + pv[1]) + (pv[2] + pv[3]);
-                lsb += (pv[4] + pv[5]) + (pv[6] + pv[7]);
-                pk[c8 * 4 + 0] = pack_bf16(pv[0], pv[1]); pk[c8 * 4 + 1] = pack_bf16(pv[2], pv[3]);
-                pk[c8 * 4 + 2] = pack_bf16(pv[4], pv[5]); pk[c8 * 4 + 3] = pack_bf16(pv[6], pv[7]);
-            }
-            tmem_st16(tp + hh * 16, pk);
-        }
-        lrun += lsa + lsb;
-        // Tree tiles are gathered by the stream two and four tiles ahead of their use, where the stage half is free
-        // and this tile's P-written arrival publishes the stores before the issuing threads need them: V of tile
-        // i + 2 (after O += P V of tile i - 2), K of tile i + 4 (its stage's K was read by S of tile i, complete).
-        if (gather_v) {
-            gather_tree(i + 2, row, UM_ROWS_THREADS, 0, false, true);
-            gather_tree(i + 2, row, UM_ROWS_THREADS, 4, false, true);
-        }
-        if (i + UM_STAGES < ntiles && i + UM_STAGES >= np) {
-            gather_tree(i + UM_STAGES, row, UM_ROWS_THREADS, 0, true, false);
-            gather_tree(i + UM_STAGES, row, UM_ROWS_THREADS, 4, true, false);
-        }
+        // P stays in tensor memory (the A operand of O += P V): this row's 64 bf16 values are 32 columns of its lane
+        tmem_st32(tP + half * (ATT_BN / 2) + lane_off, reinterpret_cast<unsigned int*>(pk));
         tmem_wait_st();
         if (i + UM_STAGES >= np) fence_proxy_async_smem();   // gathered tree tiles (generic stores) -> tensor cores
         tc_fence_before_sync();
-        // (this barrier's previous phase collected the arrivals of tile i - 4, all made before O += P V of that tile
-        // was issued, which this thread has seen complete)
-        mbar_arrive(bar_p + (i & 3) * 8);
+        mbar_arrive(bar_p + half * 8);
     }
     if (ntiles > 0 && warp < 8) mbar_wait(bar_done, 0u, p.err);
     __syncwarp();                                        // the issuing and producer warps reconverge (warp-aligned barriers follow)
