@@ -1,8 +1,12 @@
 // hs_entropy_quantify: one launch.
 //
-// Stage 1 (every CTA): a CTA owns one chunk of one logits row, loads it with 16-byte coalesced
-// loads that are all issued before the first use, and reduces max / sum e^x / sum x e^x with warp
-// shuffles.  The Top-K of the chunk is found without sorting: the K-th largest of 32 group maxima
+// Stage 1 (every CTA): a CTA owns one chunk of one logits row (up to 32 KiB), brings it on chip in
+// one piece and reduces max / sum e^x / sum x e^x with warp shuffles.  Staged variant (the default):
+// one bulk copy into shared memory, issued by one thread before the dependency wait; the passes read
+// shared memory, so a thread needs few registers and four CTAs share an SM (at one tree every CTA of
+// the launch is resident at once: no row waits for a second wave).  Register variant (rows whose
+// address or stride is not 16-byte aligned for the bulk copy; the allocation-free entry point):
+// 16-byte coalesced loads that are all issued before the first use, two CTAs per SM.  The Top-K of the chunk is found without sorting: the K-th largest of 32 group maxima
 // is a lower bound of the chunk's K-th largest logit, only threads whose own maximum reaches it
 // re-scan their registers, and the few candidates are ranked by counting.
 // Stage 2 (last CTA of a row to arrive): merges the row's chunk partials into max, log-sum-exp,
@@ -38,6 +42,7 @@ struct QuantParams {
     int* row_cnt;
     int* tree_cnt;
     int K, d_base, phi_mode, pstar_mode, entropy_mode, is_bf16;
+    int* err;        // sticky device error word (a bounded wait that expired)
 };
 
 template <bool BF16>
@@ -105,10 +110,12 @@ __device__ __noinline__ void topk_by_rounds(const char* rowp, int v0, int v1, in
 
 __device__ void tree_scores(const QuantParams& p, int b, float* s_f, int* s_i);
 
-template <bool BF16>
-__global__ void __launch_bounds__(HS_ROW_THREADS, 2) quantify_kernel(const QuantParams p) {
+template <bool BF16, bool STAGED>
+__global__ void __launch_bounds__(HS_ROW_THREADS, STAGED ? 4 : 2) quantify_kernel(const QuantParams p) {
     constexpr int VE = BF16 ? 8 : 4;
     constexpr int VPT = HS_ROW_VPT;
+    extern __shared__ __align__(16) unsigned char s_stage[];   // STAGED: the chunk, HS_ROW_THREADS * VPT vectors
+    __shared__ unsigned long long s_bar;
     __shared__ unsigned long long s_cand[CAND_CAP];
     __shared__ unsigned long long s_top[HS_MAX_TOPK];
     __shared__ unsigned long long s_red[8];
@@ -127,27 +134,47 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 2) quantify_kernel(const Quant
     if (tid < HS_MAX_TOPK) s_top[tid] = 0ull;
     if (tid == 0) s_cnt = 0;
 
-    // ---- all loads first ------------------------------------------------------------------
-    uint4 d[VPT];
-#pragma unroll
-    for (int j = 0; j < VPT; ++j) {
-        int v = v0 + tid + j * HS_ROW_THREADS;
-        if (v < v1) {
-            d[j] = __ldcs((const uint4*)(rowp) + v);
-        } else {
-            unsigned int ninf = BF16 ? 0xff80ff80u : 0xff800000u;
-            d[j] = make_uint4(ninf, ninf, ninf, ninf);
+    // ---- the chunk comes on chip: one bulk copy (STAGED) or all loads first ---------------------------
+    const unsigned int ninf = BF16 ? 0xff80ff80u : 0xff800000u;
+    uint4 d[STAGED ? 1 : VPT];
+    const uint4* sv = reinterpret_cast<const uint4*>(s_stage);
+    if (STAGED) {
+        const unsigned int bar = smem_u32(&s_bar);
+        if (tid == 0) {
+            mbar_init(bar, 1);
+            mbar_init_fence();
+            const unsigned int bytes = (unsigned int)max(v1 - v0, 0) * 16u;
+            mbar_expect_tx(bar, bytes);
+            if (bytes) bulk_load(smem_u32(s_stage), (const uint4*)(rowp) + v0, bytes, bar);
         }
+        pdl_launch_dependents();
+        pdl_wait();        // the copy above is in flight; partials and outputs may still be in use upstream
+        __syncthreads();   // the barrier is initialised
+        mbar_wait(bar, 0u, p.err);
+    } else {
+#pragma unroll
+        for (int j = 0; j < VPT; ++j) {
+            int v = v0 + tid + j * HS_ROW_THREADS;
+            d[STAGED ? 0 : j] = (v < v1) ? __ldcs((const uint4*)(rowp) + v) : make_uint4(ninf, ninf, ninf, ninf);
+        }
+        pdl_launch_dependents();
+        pdl_wait();        // the loads above are in flight; partials and outputs may still be in use upstream
     }
-    pdl_launch_dependents();
-    pdl_wait();            // the loads above are in flight; partials and outputs may still be in use upstream
+    // vector j of this thread: from shared memory or from its registers
+    auto vec = [&](int j) -> uint4 {
+        if (STAGED) {
+            const int v = tid + j * HS_ROW_THREADS;
+            return (v0 + v < v1) ? sv[v] : make_uint4(ninf, ninf, ninf, ninf);
+        }
+        return d[STAGED ? 0 : j];
+    };
     // ---- maxima ---------------------------------------------------------------------------
     float vmax[VPT];
     float tmax = -CUDART_INF_F;
 #pragma unroll
     for (int j = 0; j < VPT; ++j) {
         float x[8];
-        unpack<BF16>(d[j], x);
+        unpack<BF16>(vec(j), x);
         int v = v0 + tid + j * HS_ROW_THREADS;
         if (v == p.nvec - 1) {                       // the row's last vector may run past vocab
 #pragma unroll
@@ -166,7 +193,7 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 2) quantify_kernel(const Quant
 #pragma unroll
     for (int j = 0; j < VPT; ++j) {
         float x[8];
-        unpack<BF16>(d[j], x);
+        unpack<BF16>(vec(j), x);
         int v = v0 + tid + j * HS_ROW_THREADS;
         if (v == p.nvec - 1) {
 #pragma unroll
@@ -219,7 +246,7 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 2) quantify_kernel(const Quant
         for (int j = 0; j < VPT; ++j) {
             if (vmax[j] >= tau) {
                 float x[8];
-                unpack<BF16>(d[j], x);
+                unpack<BF16>(vec(j), x);
                 int base = (v0 + tid + j * HS_ROW_THREADS) * VE;
 #pragma unroll
                 for (int e = 0; e < VE; ++e) {
@@ -435,10 +462,21 @@ hs_status hs_launch_quantify(hs_ctx* ctx, const hs_tree_batch* tree, const void*
     p.pstar_mode = policy->pstar_mode;
     p.entropy_mode = policy->entropy_mode;
     p.is_bf16 = dtype == HS_BF16;
+    p.err = ctx->counters + HS_CNT_ERROR;
     dim3 grid(p.chunks, p.rows);
-    cudaError_t e = dtype == HS_BF16
-        ? hs_launch(quantify_kernel<true>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p)
-        : hs_launch(quantify_kernel<false>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p);
+    // the bulk copy wants 16-byte aligned rows
+    const size_t esz = dtype == HS_BF16 ? 2 : 4;
+    const bool staged = ((uintptr_t)logits % 16 == 0) && ((size_t)row_stride * esz % 16 == 0);
+    const size_t stage_bytes = (size_t)HS_ROW_THREADS * HS_ROW_VPT * 16;
+    cudaError_t e;
+    if (staged)
+        e = dtype == HS_BF16
+            ? hs_launch(quantify_kernel<true, true>, grid, dim3(HS_ROW_THREADS), stage_bytes, stream, ctx->pdl, dim3(1, 1, 1), p)
+            : hs_launch(quantify_kernel<false, true>, grid, dim3(HS_ROW_THREADS), stage_bytes, stream, ctx->pdl, dim3(1, 1, 1), p);
+    else
+        e = dtype == HS_BF16
+            ? hs_launch(quantify_kernel<true, false>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p)
+            : hs_launch(quantify_kernel<false, false>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p);
     return e == cudaSuccess ? HS_OK : HS_ERR_CUDA;
 }
 
@@ -524,7 +562,8 @@ extern "C" hs_status hs_entropy_quantify_static(const hs_tree_batch* tree, const
     // The array keeps whatever the previous call left: the arrival counters must start at zero.
     HS_CUDA_OK(cudaMemsetAsync(base, 0, HS_STATIC_COUNTER_BYTES, stream));
     dim3 grid(p.chunks, p.rows);
-    if (dtype == HS_BF16) quantify_kernel<true><<<grid, HS_ROW_THREADS, 0, stream>>>(p);
-    else quantify_kernel<false><<<grid, HS_ROW_THREADS, 0, stream>>>(p);
+    p.err = nullptr;       // (the register variant has no bounded wait)
+    if (dtype == HS_BF16) quantify_kernel<true, false><<<grid, HS_ROW_THREADS, 0, stream>>>(p);
+    else quantify_kernel<false, false><<<grid, HS_ROW_THREADS, 0, stream>>>(p);
     return cudaGetLastError() == cudaSuccess ? HS_OK : HS_ERR_CUDA;
 }
