@@ -50,6 +50,8 @@ struct AcceptParams {
     uint4* partials;      // [2][max_rows][chunks] {key lo, key hi, max, sum}
     int* row_cnt;
     int* seq_cnt;         // [batch] merged target rows of a sequence (zero between launches)
+    int staged;           // the walk may stage row slices in shared memory by bulk copies (16-byte aligned rows)
+    int* err;             // sticky device error word (a bounded wait that expired)
 };
 
 __device__ __forceinline__ float ex2a(float x) {
@@ -280,24 +282,29 @@ __device__ __forceinline__ float load_logit(const void* base, int is_bf16, size_
     return is_bf16 ? __bfloat162float(((const __nv_bfloat16*)base)[off]) : ((const float*)base)[off];
 }
 
+// This CTA's slice of the current node's target row p and draft row q: vectors [v0, v0 + nv) of the row, read
+// through pointers to shared memory (staged by bulk copies) or to the rows themselves.
+struct RowSlice {
+    const uint4* p;
+    const uint4* q;       // NULL when only p is there
+    int v0, nv;
+};
+
 // Sum over this CTA's share of the vocabulary of max(p_v - c q_v, 0), then over the cluster.
 // Every CTA returns the same value (fixed summation order).
-__device__ double cluster_residual_sum(const AcceptParams& p, cg::cluster_group& cluster, const char* prow,
-                                       const char* qrow, float pm, float ips, float qm, float iqs, float invT,
+__device__ double cluster_residual_sum(const AcceptParams& p, cg::cluster_group& cluster, const RowSlice& rs,
+                                       float pm, float ips, float qm, float iqs, float invT,
                                        float c, double* s_part, double* s_cta) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int ve = p.is_bf16 ? 8 : 4;
-    const unsigned int rank = cluster.block_rank();
-    const int per = (p.nvec + WALK_CLUSTER - 1) / WALK_CLUSTER;
-    const int v0 = rank * per, v1 = min(v0 + per, p.nvec);
     float acc = 0.f;
-    for (int v = v0 + tid; v < v1; v += WALK_THREADS) {
-        uint4 a = __ldg((const uint4*)prow + v), bq = __ldg((const uint4*)qrow + v);
+    for (int v = tid; v < rs.nv; v += WALK_THREADS) {
+        uint4 a = rs.p[v], bq = rs.q[v];
         float x[8], y[8];
         if (p.is_bf16) { unpack_v<true>(a, x); unpack_v<true>(bq, y); }
         else { unpack_v<false>(a, x); unpack_v<false>(bq, y); }
         for (int e = 0; e < ve; ++e) {
-            if (v * ve + e < p.vocab) {
+            if ((rs.v0 + v) * ve + e < p.vocab) {
                 float pv = exp2f((fmaxf(x[e], -1e30f) - pm) * invT) * ips;
                 float qv = exp2f((fmaxf(y[e], -1e30f) - qm) * invT) * iqs;
                 acc += fmaxf(pv - c * qv, 0.f);
@@ -320,20 +327,21 @@ __device__ double cluster_residual_sum(const AcceptParams& p, cg::cluster_group&
 }
 
 // Inverse-CDF draw from max(p - c q, 0) in token order: smallest j whose running sum exceeds
-// u * total; if rounding leaves none, the last token with positive mass.  `qrow` may be NULL (c = 0).
-__device__ int cluster_inverse_cdf(const AcceptParams& p, cg::cluster_group& cluster, const char* prow,
-                                   const char* qrow, float pm, float ips, float qm, float iqs, float invT,
+// u * total; if rounding leaves none, the last token with positive mass.  rs.q may be NULL (c = 0).
+// A CTA covers the tokens of its slice, a thread a contiguous run of them; running sums in double.
+__device__ int cluster_inverse_cdf(const AcceptParams& p, cg::cluster_group& cluster, const RowSlice& rs,
+                                   float pm, float ips, float qm, float iqs, float invT,
                                    float c, float u, double* s_scan, double* s_cta, int* s_pick) {
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned int rank = cluster.block_rank();
-    const int per_cta = (p.vocab + WALK_CLUSTER - 1) / WALK_CLUSTER;
-    const int c0 = rank * per_cta, c1 = min(c0 + per_cta, p.vocab);
-    const int seg = (per_cta + WALK_THREADS - 1) / WALK_THREADS;
+    const int ve = p.is_bf16 ? 8 : 4;
+    const int c0 = rs.v0 * ve, c1 = min(c0 + rs.nv * ve, p.vocab);
+    const int seg = (max(c1 - c0, 0) + WALK_THREADS - 1) / WALK_THREADS;
     const int t0 = min(c0 + tid * seg, c1), t1 = min(t0 + seg, c1);
     auto mass = [&](int j) -> float {
-        float pv = exp2f((fmaxf(load_logit(prow, p.is_bf16, j), -1e30f) - pm) * invT) * ips;
-        if (qrow == nullptr) return pv;
-        float qv = exp2f((fmaxf(load_logit(qrow, p.is_bf16, j), -1e30f) - qm) * invT) * iqs;
+        float pv = exp2f((fmaxf(load_logit(rs.p, p.is_bf16, j - c0), -1e30f) - pm) * invT) * ips;
+        if (rs.q == nullptr) return pv;
+        float qv = exp2f((fmaxf(load_logit(rs.q, p.is_bf16, j - c0), -1e30f) - qm) * invT) * iqs;
         return fmaxf(pv - c * qv, 0.f);
     };
     double mine = 0.0;
@@ -343,14 +351,24 @@ __device__ int cluster_inverse_cdf(const AcceptParams& p, cg::cluster_group& clu
         mine += (double)r;
         if (r > 0.f) last_pos = j;
     }
-    s_scan[tid] = mine;
     if (tid == 0) { s_pick[0] = 0x7fffffff; s_pick[1] = -1; }
-    __syncthreads();
-    if (tid == 0) {                       // serial exclusive scan over the CTA's threads (512 adds)
-        double run = 0.0;
-        for (int i = 0; i < WALK_THREADS; ++i) { double v = s_scan[i]; s_scan[i] = run; run += v; }
-        *s_cta = run;
+    // exclusive scan over the CTA's threads: inclusive shuffle scan inside a warp, then the warps' totals in order
+    double incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double up = __shfl_up_sync(HS_FULL_MASK, incl, o);
+        if (lane >= o) incl += up;
     }
+    if (lane == 31) s_scan[warp] = incl;
+    __syncthreads();
+    double wbefore = 0.0, ctot = 0.0;
+#pragma unroll
+    for (int w = 0; w < WALK_THREADS / 32; ++w) {
+        const double t = s_scan[w];
+        if (w < warp) wbefore += t;
+        ctot += t;
+    }
+    if (tid == 0) *s_cta = ctot;
     cluster.sync();
     double before = 0.0, total = 0.0;
     for (unsigned int r = 0; r < WALK_CLUSTER; ++r) {
@@ -359,7 +377,7 @@ __device__ int cluster_inverse_cdf(const AcceptParams& p, cg::cluster_group& clu
         total += v;
     }
     const double goal = (double)u * total;
-    double run = before + s_scan[tid];
+    double run = before + wbefore + (incl - mine);
     if (run <= goal && run + mine > goal) {          // the crossing lies in this thread's segment
         for (int j = t0; j < t1; ++j) {
             run += (double)mass(j);
@@ -382,8 +400,10 @@ __device__ int cluster_inverse_cdf(const AcceptParams& p, cg::cluster_group& clu
 __global__ void __cluster_dims__(WALK_CLUSTER, 1, 1) __launch_bounds__(WALK_THREADS)
 accept_walk_kernel(const AcceptParams p) {
     cg::cluster_group cluster = cg::this_cluster();
+    extern __shared__ __align__(16) unsigned char s_rows[];    // staged: this CTA's slices of p and q, `per` vectors each
+    __shared__ unsigned long long s_bar;
     __shared__ double s_part[WALK_THREADS / 32];
-    __shared__ double s_scan[WALK_THREADS];
+    __shared__ double s_scan[WALK_THREADS / 32];
     __shared__ double s_cta;
     __shared__ int s_pick[2];
     __shared__ int s_child;
@@ -414,6 +434,44 @@ accept_walk_kernel(const AcceptParams p) {
         }
         return;
     }
+    // This CTA's slice of a row: vectors [v0, v0 + nv).  The rows of the node the walk stands on are brought into
+    // shared memory once (one bulk copy each, only when a residual or the final draw needs them) and serve every
+    // rejection at that node and the final draw.
+    const int per = (p.nvec + WALK_CLUSTER - 1) / WALK_CLUSTER;
+    RowSlice rs;
+    rs.v0 = rank * per;
+    rs.nv = max(min(rs.v0 + per, p.nvec) - rs.v0, 0);
+    rs.p = nullptr; rs.q = nullptr;
+    const unsigned int bar = smem_u32(&s_bar);
+    if (tid == 0 && p.staged) { mbar_init(bar, 1); mbar_init_fence(); }
+    unsigned int stage_n = 0;
+    int staged_node = -1;
+    bool staged_q = false;
+    auto stage = [&](int node, const char* prow, const char* qrow) {      // qrow may be NULL: only p
+        if (staged_node == node && (staged_q || qrow == nullptr)) {
+            if (qrow == nullptr) rs.q = nullptr;
+            return;
+        }
+        staged_node = node; staged_q = qrow != nullptr;
+        if (!p.staged) {
+            rs.p = (const uint4*)prow + rs.v0;
+            rs.q = qrow ? (const uint4*)qrow + rs.v0 : nullptr;
+            return;
+        }
+        __syncthreads();                   // nobody still reads the rows of the previous node
+        if (tid == 0) {
+            const unsigned int bytes = (unsigned int)rs.nv * 16u;
+            mbar_expect_tx(bar, qrow ? 2u * bytes : bytes);
+            if (bytes) {
+                bulk_load(smem_u32(s_rows), (const uint4*)prow + rs.v0, bytes, bar);
+                if (qrow) bulk_load(smem_u32(s_rows) + (unsigned int)per * 16u, (const uint4*)qrow + rs.v0, bytes, bar);
+            }
+        }
+        mbar_wait(bar, stage_n & 1u, p.err);
+        ++stage_n;
+        rs.p = (const uint4*)s_rows;
+        rs.q = qrow ? (const uint4*)s_rows + per : nullptr;
+    };
     __syncthreads();
     int cur = 0, len = 0, bonus = -1;
     {
@@ -452,7 +510,8 @@ accept_walk_kernel(const AcceptParams p) {
                 const float u = p.uniforms ? p.uniforms[nbase + orig] : philox_uniform(p.seed, p.offset, b, orig, 0);
                 if (u < a) { accepted = j; break; }
                 const float c_next = c + (float)W;
-                const double W_next = cluster_residual_sum(p, cluster, prow, qrow, pm, ips, qm, iqs, invT,
+                stage(cur, prow, qrow);
+                const double W_next = cluster_residual_sum(p, cluster, rs, pm, ips, qm, iqs, invT,
                                                            c_next, s_part, &s_cta);
                 if (!(W_next > 0.0)) { c = 0.f; W = 1.0; tested = false; break; }   // p == q: fall back to p
                 c = c_next; W = W_next;
@@ -465,7 +524,8 @@ accept_walk_kernel(const AcceptParams p) {
                 continue;
             }
             const float ufin = p.uniforms ? p.uniforms[p.n_nodes_total + b] : philox_uniform(p.seed, p.offset, b, 0, 1);
-            bonus = cluster_inverse_cdf(p, cluster, prow, (tested && c > 0.f) ? qrow : nullptr, pm, ips, qm, iqs,
+            stage(cur, prow, (tested && c > 0.f) ? qrow : nullptr);
+            bonus = cluster_inverse_cdf(p, cluster, rs, pm, ips, qm, iqs,
                                         invT, c, ufin, s_scan, &s_cta, s_pick);
             break;
         }
@@ -529,6 +589,8 @@ hs_status hs_launch_accept(hs_ctx* ctx, const hs_tree_batch* tree, const hs_prun
     if (o > ctx->scratch_bytes) return HS_ERR_WORKSPACE;
     p.row_cnt = ctx->counters + HS_CNT_ACC_ROW;
     p.seq_cnt = ctx->counters + HS_CNT_ACC_SEQ;
+    p.err = ctx->counters + HS_CNT_ERROR;
+    p.staged = 0;
     // without draft logits every sequence must be greedy: no draft rows to scan and no sampling walk
     dim3 grid(p.chunks, rows, p.have_draft ? 2 : 1);
     cudaError_t e = dtype == HS_BF16
@@ -536,8 +598,20 @@ hs_status hs_launch_accept(hs_ctx* ctx, const hs_tree_batch* tree, const hs_prun
         : hs_launch(accept_rows_kernel<false>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p);
     if (e != cudaSuccess) return HS_ERR_CUDA;
     if (!p.have_draft) return HS_OK;
-    // the cluster shape of the walk is fixed at compile time (__cluster_dims__)
-    e = hs_launch(accept_walk_kernel, dim3(p.batch * WALK_CLUSTER), dim3(WALK_THREADS), 0, stream, ctx->pdl,
-                  dim3(1, 1, 1), p);
+    // the cluster shape of the walk is fixed at compile time (__cluster_dims__); its two row slices in shared memory
+    const size_t esz = dtype == HS_BF16 ? 2 : 4;
+    const size_t walk_smem = 2 * (size_t)((p.nvec + WALK_CLUSTER - 1) / WALK_CLUSTER) * 16;
+    p.staged = ((uintptr_t)p.target % 16 == 0) && ((uintptr_t)p.draft % 16 == 0) && ((size_t)row_stride * esz % 16 == 0) &&
+               walk_smem <= 160 * 1024;
+    static bool walk_attr[64];               // per device: the kernel may use more than 48 KiB of shared memory
+    if (ctx->device >= 0 && ctx->device < 64 && !walk_attr[ctx->device]) {
+        if (cudaFuncSetAttribute(accept_walk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024) != cudaSuccess)
+            return HS_ERR_CUDA;
+        walk_attr[ctx->device] = true;
+    } else if (ctx->device < 0 || ctx->device >= 64) {
+        p.staged = 0;
+    }
+    e = hs_launch(accept_walk_kernel, dim3(p.batch * WALK_CLUSTER), dim3(WALK_THREADS), p.staged ? walk_smem : 0, stream,
+                  ctx->pdl, dim3(1, 1, 1), p);
     return e == cudaSuccess ? HS_OK : HS_ERR_CUDA;
 }
