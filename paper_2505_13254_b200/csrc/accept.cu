@@ -291,12 +291,16 @@ struct RowSlice {
 };
 
 // Sum over this CTA's share of the vocabulary of max(p_v - c q_v, 0), then over the cluster.
-// Every CTA returns the same value (fixed summation order).
+// Every CTA returns the same value (fixed summation order).  The CTAs' sums are exchanged through s_cta[xch & 1]:
+// the buffers alternate from one exchange to the next, so one cluster barrier per exchange is enough (a buffer is
+// written again only two exchanges later, after a barrier that every CTA reaches with its reads done).
 __device__ double cluster_residual_sum(const AcceptParams& p, cg::cluster_group& cluster, const RowSlice& rs,
                                        float pm, float ips, float qm, float iqs, float invT,
-                                       float c, double* s_part, double* s_cta) {
+                                       float c, double* s_part, double* s_cta2, unsigned int& xch) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int ve = p.is_bf16 ? 8 : 4;
+    double* s_cta = s_cta2 + (xch & 1u);
+    ++xch;
     float acc = 0.f;
     for (int v = tid; v < rs.nv; v += WALK_THREADS) {
         uint4 a = rs.p[v], bq = rs.q[v];
@@ -322,7 +326,6 @@ __device__ double cluster_residual_sum(const AcceptParams& p, cg::cluster_group&
     cluster.sync();
     double tot = 0.0;
     for (unsigned int r = 0; r < WALK_CLUSTER; ++r) tot += *cluster.map_shared_rank(s_cta, r);
-    cluster.sync();                     // nobody overwrites s_cta before all have read it
     return tot;
 }
 
@@ -331,9 +334,11 @@ __device__ double cluster_residual_sum(const AcceptParams& p, cg::cluster_group&
 // A CTA covers the tokens of its slice, a thread a contiguous run of them; running sums in double.
 __device__ int cluster_inverse_cdf(const AcceptParams& p, cg::cluster_group& cluster, const RowSlice& rs,
                                    float pm, float ips, float qm, float iqs, float invT,
-                                   float c, float u, double* s_scan, double* s_cta, int* s_pick) {
+                                   float c, float u, double* s_scan, double* s_cta2, unsigned int& xch, int* s_pick) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned int rank = cluster.block_rank();
+    double* s_cta = s_cta2 + (xch & 1u);
+    ++xch;
     const int ve = p.is_bf16 ? 8 : 4;
     const int c0 = rs.v0 * ve, c1 = min(c0 + rs.nv * ve, p.vocab);
     const int seg = (max(c1 - c0, 0) + WALK_THREADS - 1) / WALK_THREADS;
@@ -404,7 +409,8 @@ accept_walk_kernel(const AcceptParams p) {
     __shared__ unsigned long long s_bar;
     __shared__ double s_part[WALK_THREADS / 32];
     __shared__ double s_scan[WALK_THREADS / 32];
-    __shared__ double s_cta;
+    __shared__ double s_cta[2];
+    unsigned int xch = 0;                  // exchanges through s_cta so far
     __shared__ int s_pick[2];
     __shared__ int s_child;
     const int tid = threadIdx.x;
@@ -512,7 +518,7 @@ accept_walk_kernel(const AcceptParams p) {
                 const float c_next = c + (float)W;
                 stage(cur, prow, qrow);
                 const double W_next = cluster_residual_sum(p, cluster, rs, pm, ips, qm, iqs, invT,
-                                                           c_next, s_part, &s_cta);
+                                                           c_next, s_part, s_cta, xch);
                 if (!(W_next > 0.0)) { c = 0.f; W = 1.0; tested = false; break; }   // p == q: fall back to p
                 c = c_next; W = W_next;
             }
@@ -526,7 +532,7 @@ accept_walk_kernel(const AcceptParams p) {
             const float ufin = p.uniforms ? p.uniforms[p.n_nodes_total + b] : philox_uniform(p.seed, p.offset, b, 0, 1);
             stage(cur, prow, (tested && c > 0.f) ? qrow : nullptr);
             bonus = cluster_inverse_cdf(p, cluster, rs, pm, ips, qm, iqs,
-                                        invT, c, ufin, s_scan, &s_cta, s_pick);
+                                        invT, c, ufin, s_scan, s_cta, xch, s_pick);
             break;
         }
     }

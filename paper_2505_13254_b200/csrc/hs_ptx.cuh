@@ -199,15 +199,6 @@ __device__ __forceinline__ void tmem_st32(unsigned int taddr, const unsigned int
         : "memory");
 }
 
-__device__ __forceinline__ void tmem_st16(unsigned int taddr, const unsigned int* r) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-        : "memory");
-}
-
 // ---- thread-block clusters: distributed shared memory -------------------------------------------------
 // shared::cluster address of `local_addr` (a shared::cta address of this CTA's window) in CTA `rank`
 __device__ __forceinline__ unsigned int cluster_map_addr(unsigned int local_addr, unsigned int rank) {

@@ -423,11 +423,11 @@ tree_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, co
 #define UM_THREADS 352                               // two softmax warpgroups + P V issuer, TMA producer, S issuer warps
 #define UM_ROWS_THREADS 128
 #define UM_SM_THREADS 256                            // softmax threads: row = tid & 127, stream = tid >> 7
-#define UM_P_BYTES (ATT_BM * ATT_BN * 2)             // 16 KiB: P tile, 128 rows x 64 keys bf16
+#define UM_MAP_BYTES 1024                            // output-row map of the rows a CTA merges (<= 65 rows x 8 bytes)
 #define UM_TMEM_COLS 512                             // S of stream g: columns 64 g ..; O: 128 + 128 g ..; P (bf16 pairs): 384 + 32 g ..
 #define UM_STAGES 4
 #define UM_RECV_BYTES (76 * 1024)                    // after the tile loop: partials pushed by the splits of the cluster
-#define UM_SMEM_BYTES (UM_STAGES * ATT_STAGE_BYTES + ATT_Q_BYTES + 2 * UM_P_BYTES + 4096 + 1024)
+#define UM_SMEM_BYTES (UM_STAGES * ATT_STAGE_BYTES + ATT_Q_BYTES + UM_MAP_BYTES + 4096 + 1024)
 
 __global__ void __launch_bounds__(UM_THREADS, 1)
 tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV) {
@@ -441,20 +441,20 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     const unsigned int smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const unsigned int sQ = smem_base + UM_STAGES * ATT_STAGE_BYTES;
-    const unsigned int sP = sQ + ATT_Q_BYTES;
+    const unsigned int sM = sQ + ATT_Q_BYTES;                // row map, then barriers and exchange arrays
     // barriers: K-full[UM_STAGES], V-full[UM_STAGES], K-free[UM_STAGES], V-free[UM_STAGES], S-ready[2],
     // partials-received, all-MMAs-done, P-written[2], S-read[2]; then the tensor-memory base.  A parity wait can only tell the
     // current phase from the one before, so every barrier is laid out such that its next completion depends on the
     // thread that waits: a stage's barriers complete once per UM_STAGES tiles, S-ready and P-written alternate with
     // the tile's parity.
-    const unsigned int bar0 = sP + 2 * UM_P_BYTES, bar_v = bar0 + UM_STAGES * 8, bar_ek = bar_v + UM_STAGES * 8,
+    const unsigned int bar0 = sM + UM_MAP_BYTES, bar_v = bar0 + UM_STAGES * 8, bar_ek = bar_v + UM_STAGES * 8,
                        bar_ev = bar_ek + UM_STAGES * 8;
     const unsigned int bar_s = bar_ev + UM_STAGES * 8, bar_r = bar_s + 16, bar_done = bar_r + 8,
                        bar_p = bar_done + 8, bar_sr = bar_p + 16, tslot = bar_sr + 16;
     unsigned char* gQ = smem_gen + UM_STAGES * ATT_STAGE_BYTES;
-    unsigned char* gP = gQ + ATT_Q_BYTES;
-    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gP + 2 * UM_P_BYTES + (4 * UM_STAGES + 8) * 8);
-    float* s_mx = reinterpret_cast<float*>(gP + 2 * UM_P_BYTES + 1024);      // [2][128]: the streams' row maxima at the end
+    unsigned char* gM = gQ + ATT_Q_BYTES;
+    volatile unsigned int* tslot_gen = reinterpret_cast<volatile unsigned int*>(gM + UM_MAP_BYTES + (4 * UM_STAGES + 8) * 8);
+    float* s_mx = reinterpret_cast<float*>(gM + UM_MAP_BYTES + 1024);      // [2][128]: the streams' row maxima at the end
     float* s_lx = s_mx + 2 * ATT_BM;                                     // [2][128]: the streams' row sums
 
     // ---- before the dependency wait: barriers, tensor memory, the first KV prefix tiles -----------------
@@ -836,7 +836,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         const unsigned int s_recv = smem_base, s_stage = smem_base + UM_RECV_BYTES;
         const int rows_max = (ATT_BM + ns - 1) / ns + 1;
         const int r_lo = (split * ATT_BM + ns - 1) / ns, r_hi = ((split + 1) * ATT_BM + ns - 1) / ns;   // rows this CTA owns
-        long long* s_og = reinterpret_cast<long long*>(gP);               // (P buffers are idle now)                          // output row of each owned row (or -1)
+        long long* s_og = reinterpret_cast<long long*>(gM);               // output row of each owned row (or -1)
         if (tid == 0) mbar_expect_tx(bar_r, (unsigned int)(ns * (r_hi - r_lo) * ATT_PO_STRIDE * 4));
         if (tid < r_hi - r_lo) {
             const int rg = m0 + r_lo + tid;
