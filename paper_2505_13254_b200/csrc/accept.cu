@@ -23,7 +23,7 @@
 namespace cg = cooperative_groups;
 
 #define LOG2E 1.4426950408889634f
-#define WALK_CLUSTER 8
+#define WALK_CLUSTER 16       // (larger than the portable 8: the launcher asks for it)
 #define WALK_THREADS 512
 
 struct RowOut {           // per kept node, in the workspace
@@ -611,7 +611,8 @@ hs_status hs_launch_accept(hs_ctx* ctx, const hs_tree_batch* tree, const hs_prun
                walk_smem <= 160 * 1024;
     static bool walk_attr[64];               // per device: the kernel may use more than 48 KiB of shared memory
     if (ctx->device >= 0 && ctx->device < 64 && !walk_attr[ctx->device]) {
-        if (cudaFuncSetAttribute(accept_walk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024) != cudaSuccess)
+        if (cudaFuncSetAttribute(accept_walk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(accept_walk_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
             return HS_ERR_CUDA;
         walk_attr[ctx->device] = true;
     } else if (ctx->device < 0 || ctx->device >= 64) {
