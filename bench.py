@@ -58,6 +58,14 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def tensor_peak():
+    """Dense bf16 TFLOP/s of this machine's B200s (burst figure: the kernel is timed alone)."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        return float(json.load(open(path))["bf16_tflops"])
+    return 1590.0
+
+
 class ClockSampler:
     """nvidia-smi clocks / throttle reasons sampled while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -355,11 +363,26 @@ def main():
         "device_error_word": dev_err,
     }
     a_gbs = kern["attention"]["gbs"]
-    line["roofline_attention"] = {"kernel": "tree_attn_umma_kernel (hs_tree_verify_attention, one launch per step)",
-                                  "bound": "hbm", "achieved": a_gbs, "peak": peak, "unit": "GB/s",
-                                  "frac": a_gbs / peak if a_gbs else None, "peak_kind": peak_kind + " (burst copy figure)",
-                                  "traffic": ncu_traffic("tree_attn_umma_kernel", cfg.name),
-                                  "algorithmic_bytes_per_launch": attn_bytes}
+    # Q K^T and P V of every kept row against its sequence's prefix and tree: 4 * 128 flops per (row, key) pair
+    kv_len = np.diff(batch["kv_off"]).astype(np.int64)
+    nk_b = st.pruned.n_keep.cpu().numpy().astype(np.int64)[: len(kv_len)]
+    attn_flops = float(4 * cfg.head_dim * cfg.hq * (nk_b * (kv_len + nk_b)).sum())
+    a_tflops = attn_flops / (kern["attention"]["us"] * 1e-6) / 1e12
+    tf_peak = tensor_peak()
+    if attn_flops / (tf_peak * 1e12) > attn_bytes / (peak * 1e9):      # the tensor pipe is the longer leg
+        line["roofline_attention"] = {"kernel": "tree_attn_umma_kernel (hs_tree_verify_attention, one launch per step)",
+                                      "bound": "tensor", "achieved": a_tflops, "peak": tf_peak, "unit": "TFLOP/s",
+                                      "frac": a_tflops / tf_peak, "peak_kind": peak_kind + " (dense bf16 burst figure)",
+                                      "traffic": ncu_traffic("tree_attn_umma_kernel", cfg.name),
+                                      "algorithmic_flops_per_launch": attn_flops,
+                                      "algorithmic_bytes_per_launch": attn_bytes}
+    else:
+        line["roofline_attention"] = {"kernel": "tree_attn_umma_kernel (hs_tree_verify_attention, one launch per step)",
+                                      "bound": "hbm", "achieved": a_gbs, "peak": peak, "unit": "GB/s",
+                                      "frac": a_gbs / peak if a_gbs else None, "peak_kind": peak_kind + " (burst copy figure)",
+                                      "traffic": ncu_traffic("tree_attn_umma_kernel", cfg.name),
+                                      "algorithmic_bytes_per_launch": attn_bytes,
+                                      "algorithmic_flops_per_launch": attn_flops}
     if not args.no_cpu_baseline:
         from oracle import step as ostep
         nrep = 5
