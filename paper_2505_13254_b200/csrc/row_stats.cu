@@ -4,9 +4,9 @@
 // one piece and reduces max / sum e^x / sum x e^x with warp shuffles.  Staged variant (the default):
 // one bulk copy into shared memory, issued by one thread before the dependency wait; the passes read
 // shared memory, so a thread needs few registers and four CTAs share an SM (at one tree every CTA of
-// the launch is resident at once: no row waits for a second wave).  Register variant (rows whose
-// address or stride is not 16-byte aligned for the bulk copy; the allocation-free entry point):
-// 16-byte coalesced loads that are all issued before the first use, two CTAs per SM.  The Top-K of the chunk is found without sorting: the K-th largest of 32 group maxima
+// the launch is resident at once: no row waits for a second wave).  Register variant (the
+// allocation-free entry point, and rows a caller of the launcher hands over unaligned: the C entry
+// point rejects those): 16-byte coalesced loads that are all issued before the first use, two CTAs per SM.  The Top-K of the chunk is found without sorting: the K-th largest of 32 group maxima
 // is a lower bound of the chunk's K-th largest logit, only threads whose own maximum reaches it
 // re-scan their registers, and the few candidates are ranked by counting.
 // Stage 2 (last CTA of a row to arrive): merges the row's chunk partials into max, log-sum-exp,
