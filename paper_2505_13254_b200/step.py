@@ -104,3 +104,39 @@ class VerifyStep:
             self.attention(db)
         self.accept_path(db)
         return self
+
+
+def refill(db: DeviceBatch, batch: dict) -> None:
+    """Copies another batch of the same shapes (nodes, KV lengths, dtypes) into the device buffers of `db`."""
+    src = upload(batch, db.tree.parent.device)
+    if (src.tree.n_nodes_total, src.tree.batch, src.seed, src.offset) != \
+            (db.tree.n_nodes_total, db.tree.batch, db.seed, db.offset):
+        raise ValueError("refill needs a batch of the same shape and Philox seed / offset")
+    for a, b in ((db.tree.node_off, src.tree.node_off), (db.tree.parent, src.tree.parent), (db.tree.token, src.tree.token),
+                 (db.draft, src.draft), (db.target, src.target), (db.q, src.q), (db.k_tree, src.k_tree),
+                 (db.v_tree, src.v_tree), (db.k_cache, src.k_cache), (db.v_cache, src.v_cache), (db.kv_off, src.kv_off),
+                 (db.mode, src.mode), (db.temperature, src.temperature)):
+        if a is not None:
+            if a.shape != b.shape:
+                raise ValueError("refill needs a batch of the same shape")
+            a.copy_(b)
+
+
+class GraphedStep:
+    """The four calls over fixed input buffers, captured once into a CUDA graph and replayed (Sec. 4.3, the
+    computation graph kept ready per regime).  One graph serves every entropy bin: the kernels read d', N' and the
+    kept nodes from device memory, so nothing in the launch shapes depends on the regime.  Scalars of the calls
+    (Philox seed and offset, strides) are part of the graph; the inputs are refreshed in place (`refill`)."""
+
+    def __init__(self, step: VerifyStep, db: DeviceBatch, warmup: int = 2):
+        self.step, self.db = step, db
+        for _ in range(warmup):                       # first calls resolve attributes and tensor maps outside the capture
+            step.run(db)
+        torch.cuda.synchronize()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            step.run(db)
+
+    def replay(self) -> VerifyStep:
+        self.graph.replay()
+        return self.step

@@ -118,3 +118,27 @@ def test_alternative_readings(ctx):
         lo, hi = (0.0, 4.0) if "entropy_mode" in mode else (4.0, 12.0)
         pol["thresholds"] = list(np.linspace(lo, hi, 7))
         run_and_check(ctx, cfg, pol, 300, attention="none")
+
+
+# ---- one captured graph serves every entropy bin (Sec. 4.3) -----------------------------------------------
+
+@pytest.mark.gpu
+def test_graph_replay_across_bins(ctx):
+    cfg, base = SMALL["c2_small"]
+    policy = pu.policy_for(cfg, base)
+    cases = [pu.oracle_case(cfg, policy, seed) for seed in (2100, 2200, 2300, 2400, 2500, 2600)]
+    bins = {int(res[0]["pruned"]["bin"]) for _, res in cases}
+    assert len(bins) >= 2                      # the seeds land in different regimes (different d', N')
+    db = gstep.upload(cases[0][0])
+    st = gstep.VerifyStep(ctx, db, policy)
+    g = gstep.GraphedStep(st, db)
+    for batch, res in cases[1:] + cases[:1]:
+        batch = dict(batch, philox_seed=cases[0][0]["philox_seed"], philox_offset=cases[0][0]["philox_offset"])
+        gstep.refill(db, batch)
+        g.replay()
+        torch.cuda.synchronize()
+        pu.check_quant(st.quant, batch, res, policy["top_k"])
+        pu.check_pruned(st.pruned, res)
+        pu.check_attention(st.attn_out, st.attn_lse, batch, res)
+        pu.check_accept(st.accept, res)
+        assert hb.hs_device_error(ctx) == 0
