@@ -7,6 +7,11 @@ distribution is replaced by the normalised residual max(p - q, 0) and the next s
 is tried (the chain rule of Sec. 2.1 applied to each sibling in turn, as in tree-based
 verification); when no candidate is left the next token is drawn from the residual.
 
+Deterministic proposals (a second reading of Sec. 2.1 for drafts that propose one fixed token per
+candidate instead of a sample: the proposal distribution of candidate x is the point mass on its
+token): the same chain rule with q = point mass, so x is accepted with probability r(token of x)
+and a rejection removes that token from the residual.
+
 Inputs use the pruned ("compact") tree: parent[i] < i, node 0 the root; target[i] is the
 target model's logits row after kept node i, draft[i] the draft model's row after it.
 """
@@ -74,6 +79,49 @@ def rejection(parent, token, target, draft, temperature, u_accept, u_final, trac
                     r = p
                     break
                 r = r / z
+        if accepted is None:
+            cdf = np.cumsum(r)
+            hit = np.nonzero(cdf > u_final)[0]
+            bonus = int(hit[0]) if len(hit) else int(np.nonzero(r > 0)[0][-1])
+            if trace is not None:
+                trace.append(("final", float(u_final), float(cdf[bonus - 1]) if bonus else 0.0,
+                              float(cdf[bonus])))
+            return path, bonus
+        cur = accepted
+        path.append(cur)
+
+
+def deterministic(parent, token, target, temperature, u_accept, u_final, trace=None):
+    """Multi-candidate acceptance when every candidate is a deterministic proposal.
+
+    At node cur with p = softmax(target[cur] / T) and r = p: children are tried in index order;
+    the proposal distribution of child x is q = the point mass on tok = token[x], so x is accepted
+    iff u_accept[x] < min(1, r[tok] / q[tok]) = r[tok]; otherwise r <- normalise(max(r - q, 0)),
+    which removes tok from r.  After the last rejection (or at a leaf) the bonus token is the
+    smallest j with cumsum(r)[j] > u_final.  ``trace`` as in `rejection`.
+    """
+    path = [0]
+    cur = 0
+    while True:
+        p, _, _ = softmax64(np.asarray(target[cur], dtype=np.float64) / temperature)
+        r = p
+        accepted = None
+        for x in children_of(parent, cur):
+            t = token[x]
+            q = np.zeros_like(p)
+            q[t] = 1.0
+            a = min(1.0, r[t] / q[t])
+            if trace is not None:
+                trace.append(("accept", x, float(u_accept[x]), float(a)))
+            if u_accept[x] < a:
+                accepted = x
+                break
+            r = np.maximum(r - q, 0.0)
+            z = r.sum()
+            if z <= 0.0:                # the whole mass sat on rejected tokens: keep p
+                r = p
+                break
+            r = r / z
         if accepted is None:
             cdf = np.cumsum(r)
             hit = np.nonzero(cdf > u_final)[0]

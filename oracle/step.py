@@ -52,6 +52,12 @@ def accept_path(batch, b, pr, trace=None):
     target = _widen(batch["target"][keep])
     if batch["mode"][b] == 0:
         path, bonus = accept.greedy(pr["new_parent"], token, target)
+    elif batch["mode"][b] == 2:
+        seed, off = batch["philox_seed"], batch["philox_offset"]
+        u_acc = np.array([philox.uniform(seed, off, b, int(orig), 0) for orig in pr["keep_idx"]])
+        u_fin = philox.uniform(seed, off, b, 0, 1)
+        path, bonus = accept.deterministic(pr["new_parent"], token, target, float(batch["temperature"][b]),
+                                           u_acc, u_fin, trace=trace)
     else:
         draft = _widen(batch["draft"][keep])
         seed, off = batch["philox_seed"], batch["philox_offset"]

@@ -149,3 +149,69 @@ def test_residual_scalar_recurrence():
     cdf = np.cumsum(np.maximum(p - c * q, 0) / W)
     j = int(np.searchsorted(cdf, 0.3, side="right"))
     assert final[3] == pytest.approx(cdf[j], rel=1e-12)
+
+
+# ---- deterministic proposals (q = point mass on the candidate's token) ------------------------------------
+
+def test_deterministic_chain_equals_rejection_with_point_mass_draft():
+    """On a chain every node has one candidate, and a draft row that puts all its mass on that candidate's token
+    turns the general sampler (pinned above) into the deterministic-proposal one."""
+    rng = np.random.default_rng(11)
+    n, V = 6, 9
+    parent = np.arange(-1, n - 1)
+    for trial in range(200):
+        token = rng.integers(0, V, n)
+        target = rng.standard_normal((n, V)) * 2.0
+        draft = np.full((n, V), -1e30)
+        for i in range(n - 1):
+            draft[i, token[i + 1]] = 0.0            # softmax: the point mass on the child's token
+        draft[n - 1, 0] = 0.0
+        u, uf = rng.random(n), rng.random()
+        assert accept.deterministic(parent, token, target, 0.8, u, uf) == \
+            accept.rejection(parent, token, target, draft, 0.8, u, uf)
+
+
+def test_deterministic_closed_form_of_sibling_tests():
+    """The k-th sibling is accepted with probability p(t_k) / (1 - sum of p over the tokens rejected before it);
+    the bonus token comes from p with the rejected tokens removed."""
+    rng = np.random.default_rng(12)
+    V, k = 10, 4
+    parent = np.array([-1] + [0] * k)
+    for trial in range(200):
+        target = rng.standard_normal((k + 1, V)) * 1.5
+        p = softmax64(target[0])[0]
+        token = np.concatenate([[0], rng.choice(V, size=k, replace=False)])
+        u, uf = rng.random(k + 1), rng.random()
+        trace = []
+        path, bonus = accept.deterministic(parent, token, target, 1.0, u, uf, trace=trace)
+        gone, want = 0.0, None
+        for x in range(1, k + 1):
+            a = p[token[x]] / (1.0 - gone)
+            if u[x] < min(1.0, a):
+                want = x
+                break
+            gone += p[token[x]]
+        if want is not None:
+            assert path == [0, want]
+        else:
+            r = p.copy(); r[token[1:]] = 0.0; r /= r.sum()
+            assert path == [0] and bonus == int(np.searchsorted(np.cumsum(r), uf, side="right"))
+    # u = 0 accepts the first candidate whose token has any mass
+    path, _ = accept.deterministic(parent, token, target, 1.0, np.zeros(k + 1), 0.5)
+    assert path == [0, 1]
+
+
+def test_deterministic_lossless_output_distribution():
+    """Whatever fixed tokens the candidates carry, the token emitted after the root follows the target distribution."""
+    rng = np.random.default_rng(13)
+    V, k, trials = 8, 3, 40000
+    target = rng.standard_normal((k + 1, V)) * 1.5
+    p = softmax64(target[0])[0]
+    parent = np.array([-1] + [0] * k)
+    token = np.array([0, 5, 2, 7])                  # fixed proposals (e.g. the draft model's top-3)
+    counts = np.zeros(V)
+    for _ in range(trials):
+        path, bonus = accept.deterministic(parent, token, target, 1.0, rng.random(k + 1), rng.random())
+        counts[token[path[1]] if len(path) > 1 else bonus] += 1
+    chi2 = ((counts - trials * p) ** 2 / (trials * p)).sum()
+    assert scipy.stats.chi2.sf(chi2, V - 1) > 1e-3
