@@ -174,11 +174,15 @@ def main():
     ap.add_argument("--workload", default="c2_8b")
     ap.add_argument("--rotate", type=int, default=0, help="distinct input copies (0 = enough to exceed 2x L2)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--accept", default=None, choices=["greedy", "rejection", "mixed", "deterministic", "mixed3"],
+                    help="acceptance mode(s) of the sequences instead of the workload's own")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     from paper_2505_13254_b200 import synth
     cfg = synth.CONFIGS[args.workload]
+    if args.accept:
+        cfg = cfg.scaled(accept=args.accept, temperature=cfg.temperature or 1.0)
     if args.impl == "reference":
         if args.steps > 20:
             args.steps = 5                 # bounded: a step is seconds of CPU work

@@ -59,7 +59,10 @@ typedef enum {
 } hs_status;
 
 typedef enum { HS_F32 = 0, HS_BF16 = 1 } hs_dtype;
-typedef enum { HS_ACCEPT_GREEDY = 0, HS_ACCEPT_REJECTION = 1 } hs_accept_mode;
+/* GREEDY: Sec. 5 (temperature 0).  REJECTION: Sec. 2.1, candidates sampled from the draft distribution q.
+ * DETERMINISTIC: Sec. 2.1 with a point-mass proposal per candidate (drafts that propose fixed tokens, e.g. their
+ * top-k): candidate x is accepted with probability r(token of x), a rejection removes that token from r. */
+typedef enum { HS_ACCEPT_GREEDY = 0, HS_ACCEPT_REJECTION = 1, HS_ACCEPT_DETERMINISTIC = 2 } hs_accept_mode;
 /* Layout of per-kept-node rows (q, k_tree, v_tree, out, target logits):
  *   COMPACT  row keep_off[b] + i           belongs to kept node i of sequence b
  *   ORIGINAL row node_off[b] + keep_idx[.] belongs to it (rows indexed by drafted node id) */
@@ -208,9 +211,9 @@ hs_status hs_tree_verify_attention(hs_ctx* ctx, const hs_pruned_tree* pruned, co
 
 /* Sec. 2.1 (sampling) and Sec. 5 (temperature 0).  target_logits rows follow `target_layout`;
  * draft_logits rows are always indexed by original node id (as given to hs_entropy_quantify) and
- * are read only by sequences in rejection mode; a caller whose sequences are all greedy passes NULL
- * (a rejection-mode sequence then gets status HS_ERR_INVALID_ARG) and saves a launch.  mode[b]: hs_accept_mode; temperature[b] > 0 for
- * rejection mode, applied to both models.  Uniforms: Philox4x32-10 with key = seed, counter =
+ * are read only by sequences in rejection mode; a caller without such sequences passes NULL (a
+ * rejection-mode sequence then gets status HS_ERR_INVALID_ARG) and saves a launch.  mode[b]: hs_accept_mode;
+ * temperature[b] > 0 for the two sampling modes, applied to both models.  Uniforms: Philox4x32-10 with key = seed, counter =
  * (offset, b, original node id, stream) with stream 0 = accept test of that node, 1 = final draw
  * (node 0); u = (x0 >> 8) * 2^-24.  If `uniforms` is not NULL it overrides the generator:
  * uniforms[node_off[b] + node] for accept tests and uniforms[n_nodes_total + b] for the final draw. */

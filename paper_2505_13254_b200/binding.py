@@ -17,7 +17,7 @@ import torch
 HS_MAX_NODES = 128
 HS_MAX_TOPK = 16
 HS_F32, HS_BF16 = 0, 1
-HS_ACCEPT_GREEDY, HS_ACCEPT_REJECTION = 0, 1
+HS_ACCEPT_GREEDY, HS_ACCEPT_REJECTION, HS_ACCEPT_DETERMINISTIC = 0, 1, 2
 HS_ROWS_COMPACT, HS_ROWS_ORIGINAL = 0, 1
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libheterospec.so")

@@ -119,8 +119,185 @@ __device__ void greedy_walk(const AcceptParams& p, int b) {
     }
 }
 
+__device__ __forceinline__ float load_logit(const void* base, int is_bf16, size_t off);
+
+// Acceptance of sequence b with deterministic proposals by one whole CTA (Sec. 2.1 with a point-mass proposal per
+// candidate): at node cur with p = softmax(target row / T) the kept children are tried in index order; child x
+// with token t is accepted iff u_x < min(1, p_t / W), W = 1 - (mass of the tokens rejected at this node so far); a
+// rejection removes t.  When no candidate is left the bonus token is drawn by inverse CDF in token order from p
+// without the rejected tokens (running sums in double, one contiguous run of tokens per thread).
+__device__ __noinline__ void deterministic_walk(const AcceptParams& p, int b) {
+    __shared__ int s_par[HS_MAX_NODES], s_tok[HS_MAX_NODES], s_rej[HS_MAX_NODES];
+    __shared__ double s_scan[HS_ROW_THREADS / 32];
+    __shared__ double s_phase[64];
+    __shared__ int s_pick[2];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x;
+    const int koff = p.pr.keep_off[b];
+    const int nk = min(p.pr.n_keep[b], HS_MAX_NODES);
+    const int nbase = p.node_off[b];
+    const int cap = p.out.path_cap;
+    for (int j = tid; j < cap; j += nthr) {
+        p.out.path_nodes[b * cap + j] = -1;
+        p.out.path_compact[b * cap + j] = -1;
+        p.out.path_tokens[b * cap + j] = -1;
+    }
+    for (int j = tid; j < nk; j += nthr) {
+        s_par[j] = p.pr.new_parent[koff + j];
+        s_tok[j] = p.token[nbase + p.pr.keep_idx[koff + j]];
+    }
+    __syncthreads();
+    const float invT = LOG2E / p.temperature[b];
+    const size_t esz = p.is_bf16 ? 2 : 4;
+    int cur = 0, len = 0, bonus = -1;
+    for (int step = 0; step < nk; ++step) {
+        if (tid == 0 && len < cap) {
+            p.out.path_compact[b * cap + len] = cur;
+            p.out.path_nodes[b * cap + len] = p.pr.keep_idx[koff + cur];
+        }
+        const int orig_cur = p.pr.keep_idx[koff + cur];
+        const int trow = p.target_layout == HS_ROWS_ORIGINAL ? nbase + orig_cur : koff + cur;
+        const char* prow = (const char*)p.target + (size_t)trow * p.row_stride * esz;
+        const float2 pms = __ldcg(&p.ro.tgt_ms[koff + cur]);      // written by another CTA of this launch
+        const float pm = pms.x, ips = 1.f / pms.y;
+        double W = 1.0;
+        int nrej = 0, accepted = -1;
+        for (int j = cur + 1; j < nk; ++j) {                     // siblings in index order (every thread the same)
+            if (s_par[j] != cur) continue;
+            const int t = s_tok[j];
+            const float pt = exp2f((fmaxf(load_logit(prow, p.is_bf16, t), -1e30f) - pm) * invT) * ips;
+            const float a = fminf(1.f, pt / (float)W);
+            const int orig = p.pr.keep_idx[koff + j];
+            const float u = p.uniforms ? p.uniforms[nbase + orig] : philox_uniform(p.seed, p.offset, b, orig, 0);
+            if (u < a) { accepted = j; break; }
+            const double W_next = W - (double)pt;
+            if (!(W_next > 0.0)) { nrej = 0; W = 1.0; break; }  // nothing left: fall back to p
+            if (tid == 0) s_rej[nrej] = t;
+            ++nrej;
+            W = W_next;
+        }
+        if (accepted >= 0) {
+            if (tid == 0 && len < cap) p.out.path_tokens[b * cap + len] = s_tok[accepted];
+            cur = accepted;
+            ++len;
+            continue;
+        }
+        // ---- the bonus token: inverse CDF over the vocabulary without the rejected tokens -------------------
+        // The row is taken in phases of nthr * 4 vectors; in a phase thread t owns 4 consecutive 16-byte vectors (all
+        // loads in flight together), so token order is (phase, thread, token).  Pass 1 sums
+        // every phase; then the phase that holds the crossing is summed again and scanned.
+        const float ufin = p.uniforms ? p.uniforms[p.n_nodes_total + b] : philox_uniform(p.seed, p.offset, b, 0, 1);
+        if (tid == 0) { s_pick[0] = 0x7fffffff; s_pick[1] = -1; }
+        __syncthreads();                                         // s_rej, s_pick
+        const int ve = p.is_bf16 ? 8 : 4;
+        const int phase_vecs = nthr * 4;
+        const int nph = (p.nvec + phase_vecs - 1) / phase_vecs;  // <= 64 for vocabularies up to 2^19 bf16 (larger ones: status below)
+        // masses of this thread's 4 vectors of phase ph (0 past the vocabulary and for rejected tokens)
+        auto phase_mass = [&](int ph, float (&m)[4][8]) {
+            uint4 d[4];
+            const int vbase = ph * phase_vecs + tid * 4;
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                d[q] = (vbase + q < p.nvec) ? __ldg((const uint4*)prow + vbase + q) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                float x[8];
+                if (p.is_bf16) unpack_v<true>(d[q], x); else unpack_v<false>(d[q], x);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int tok = (vbase + q) * ve + e;
+                    const bool in = e < ve && vbase + q < p.nvec && tok < p.vocab;
+                    m[q][e] = in ? exp2f((fmaxf(x[e], -1e30f) - pm) * invT) * ips : 0.f;
+                }
+            }
+            for (int k = 0; k < nrej; ++k) {                     // few: the siblings rejected at this node
+                const int rv = s_rej[k] / ve - vbase;
+                if (rv >= 0 && rv < 4) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            if (q == rv && e == s_rej[k] % ve) m[q][e] = 0.f;
+                }
+            }
+        };
+        int last_pos = -1;
+        for (int ph = 0; ph < nph; ++ph) {
+            float m[4][8];
+            phase_mass(ph, m);
+            double mine = 0.0;
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    mine += (double)m[q][e];
+                    if (m[q][e] > 0.f) last_pos = ((ph * phase_vecs + tid * 4 + q) * ve + e);
+                }
+            const double w = warp_sum_d(mine);
+            if (lane == 0) s_scan[warp] = w;
+            __syncthreads();
+            if (tid == 0) {
+                double t = 0.0;
+                for (int w2 = 0; w2 < nthr / 32; ++w2) t += s_scan[w2];
+                s_phase[ph] = t;
+            }
+            __syncthreads();
+        }
+        double total = 0.0;
+        for (int ph = 0; ph < nph; ++ph) total += s_phase[ph];
+        const double goal = (double)ufin * total;
+        int phx = -1;                                            // first phase whose running total exceeds the goal
+        double before_ph = 0.0;
+        for (int ph = 0; ph < nph; ++ph) {
+            if (before_ph + s_phase[ph] > goal) { phx = ph; break; }
+            before_ph += s_phase[ph];
+        }
+        if (phx >= 0) {
+            float m[4][8];
+            phase_mass(phx, m);
+            double mine = 0.0;
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) mine += (double)m[q][e];
+            double incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const double up = __shfl_up_sync(HS_FULL_MASK, incl, o);
+                if (lane >= o) incl += up;
+            }
+            if (lane == 31) s_scan[warp] = incl;
+            __syncthreads();
+            double run = before_ph + (incl - mine);
+            for (int w2 = 0; w2 < warp; ++w2) run += s_scan[w2];
+            if (run <= goal && run + mine > goal) {              // the crossing lies in this thread's tokens
+                bool found = false;
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        run += (double)m[q][e];
+                        if (!found && run > goal) {
+                            found = true;
+                            atomicMin(&s_pick[0], (phx * phase_vecs + tid * 4 + q) * ve + e);
+                        }
+                    }
+            }
+        }
+        if (last_pos >= 0) atomicMax(&s_pick[1], last_pos);
+        __syncthreads();
+        bonus = s_pick[0] != 0x7fffffff ? s_pick[0] : max(s_pick[1], 0);
+        break;
+    }
+    if (tid == 0) {
+        p.out.accept_len[b] = len;
+        p.out.bonus_token[b] = bonus;
+        p.out.terminal_rank[b] = p.pr.keep_rank[koff + cur];
+        p.out.status[b] = HS_OK;
+    }
+}
+
 template <bool BF16>
-__global__ void __launch_bounds__(HS_ROW_THREADS, 4) accept_rows_kernel(const AcceptParams p) {
+__global__ void __launch_bounds__(HS_ROW_THREADS, 4) accept_rows_kernel(const __grid_constant__ AcceptParams p) {
     constexpr int VE = BF16 ? 8 : 4;
     constexpr int VPT = HS_ROW_VPT;
     __shared__ float s_w[8][2];
@@ -152,9 +329,10 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 4) accept_rows_kernel(const Ac
     const int b = lo;
     const int i = k - p.pr.keep_off[b];
     const int nk = p.pr.n_keep[b];
-    const bool sampling = p.mode[b] == HS_ACCEPT_REJECTION;
+    const int md = p.mode[b];
+    const bool sampling = md != HS_ACCEPT_GREEDY;          // the row's normaliser is needed
     if (which == 1) {
-        if (!sampling) return;
+        if (md != HS_ACCEPT_REJECTION) return;
         int internal = 0;                         // does kept node i have a kept child?
         for (int j = i + 1 + tid; j < nk; j += HS_ROW_THREADS)
             internal |= (p.pr.new_parent[p.pr.keep_off[b] + j] == i);
@@ -259,12 +437,12 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 4) accept_rows_kernel(const Ac
     }
     }
     // ---- greedy sequences finish here: the last target row of a sequence to be merged walks its tree ------
-    if (sampling && !p.have_draft && which == 0 && i == 0 && tid == 0) {
+    if (md == HS_ACCEPT_REJECTION && !p.have_draft && which == 0 && i == 0 && tid == 0) {
         // rejection sampling needs the draft distribution: the caller passed none
         p.out.accept_len[b] = 0; p.out.bonus_token[b] = -1; p.out.terminal_rank[b] = -1;
         p.out.status[b] = HS_ERR_INVALID_ARG;
     }
-    if (which != 0 || sampling) return;
+    if (which != 0 || md == HS_ACCEPT_REJECTION) return;
     __syncthreads();
     if (tid == 0) {
         __threadfence();
@@ -273,7 +451,10 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 4) accept_rows_kernel(const Ac
         __threadfence();
     }
     __syncthreads();
-    if (s_flag) greedy_walk(p, b);
+    if (s_flag) {
+        if (md == HS_ACCEPT_GREEDY) greedy_walk(p, b);
+        else deterministic_walk(p, b);
+    }
 }
 
 // ---- the walk ----------------------------------------------------------------------------------

@@ -62,7 +62,7 @@ def upload(batch: dict, device="cuda:0") -> DeviceBatch:
                        torch.from_numpy(np.asarray(batch["temperature"], dtype=np.float32)).to(device),
                        int(batch["philox_seed"]), int(batch["philox_offset"]),
                        int(np.diff(node_off).max()), int(np.diff(kv_off).max()),
-                       bool(np.any(np.asarray(batch["mode"]) != 0)))
+                       bool(np.any(np.asarray(batch["mode"]) == hb.HS_ACCEPT_REJECTION)))
 
 
 class VerifyStep:
@@ -92,7 +92,7 @@ class VerifyStep:
                                            node_off=db.tree.node_off, out=self.attn_out, lse_out=self.attn_lse)
 
     def accept_path(self, db: DeviceBatch):
-        draft = db.draft if db.any_sampling else None        # greedy-only batches need no draft rows
+        draft = db.draft if db.any_sampling else None        # only rejection-sampling sequences read draft rows
         return hb.hs_accept_path(self.ctx, db.tree, self.pruned, db.target, draft, db.mode, db.temperature,
                                  target_layout=hb.HS_ROWS_ORIGINAL, seed=db.seed, offset=db.offset,
                                  path_cap=self.accept.path_cap, out=self.accept)

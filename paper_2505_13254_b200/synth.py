@@ -73,7 +73,7 @@ class VerifyConfig:
     hkv: int
     head_dim: int
     kv_len: Tuple[int, int]           # inclusive range of prefix lengths
-    accept: str                       # "greedy" | "rejection" | "mixed"
+    accept: str                       # "greedy" | "rejection" | "mixed" | "deterministic" | "mixed3"
     temperature: float
     peaked_frac: Tuple[float, float] = (0.6, 0.6)   # per-sequence fraction of peaked rows
     boost_prob: float = 0.9
@@ -324,10 +324,14 @@ def make_batch(cfg: VerifyConfig, seed: int, with_logits: bool = True,
         mode = np.zeros(cfg.batch, dtype=np.int32)
     elif cfg.accept == "rejection":
         mode = np.ones(cfg.batch, dtype=np.int32)
+    elif cfg.accept == "deterministic":
+        mode = np.full(cfg.batch, 2, dtype=np.int32)
+    elif cfg.accept == "mixed3":
+        mode = (np.arange(cfg.batch) % 3).astype(np.int32)
     else:
         mode = (np.arange(cfg.batch) % 2).astype(np.int32)
     batch["mode"] = mode
-    batch["temperature"] = np.where(mode == 1, cfg.temperature, 0.0).astype(np.float32)
+    batch["temperature"] = np.where(mode != 0, cfg.temperature, 0.0).astype(np.float32)
     batch["philox_seed"] = (int(seed) * 0x9E3779B97F4A7C15 + 0x1234567) & (2**64 - 1)
     batch["philox_offset"] = 0
     return batch

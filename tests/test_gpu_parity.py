@@ -51,6 +51,9 @@ SMALL = {
     "c3_small": (synth.CONFIGS["c3_70b"].scaled(kv_len=(200, 200)), "c3_70b"),
     "c4_small": (synth.CONFIGS["c4_ragged"].scaled(batch=5, kv_len=(1, 400)), "c4_ragged"),
     "c5_small": (synth.CONFIGS["c5_long"].scaled(batch=2, kv_len=(700, 700)), "c5_long"),
+    # acceptance with deterministic proposals (mode 2), alone and mixed with the two other modes in one batch
+    "c3_small_det": (synth.CONFIGS["c3_70b"].scaled(kv_len=(200, 200), accept="deterministic"), "c3_70b"),
+    "c4_small_mixed3": (synth.CONFIGS["c4_ragged"].scaled(batch=6, kv_len=(1, 400), accept="mixed3"), "c4_ragged"),
 }
 
 
