@@ -5,6 +5,9 @@
 //                      over the draft row of every kept internal node of a sampling sequence.
 //                      Same register-resident 16-byte-load pattern as the entropy pass; the last
 //                      chunk of a row merges the chunk partials.
+//                      Greedy sequences and sequences with deterministic proposals finish here: the CTA
+//                      that merges a sequence's last target row walks its tree (greedy_walk,
+//                      deterministic_walk).
 // accept_walk_kernel   one thread-block cluster per sequence walks the tree from the root.
 //                      Greedy (temperature 0): follow the child whose token is the arg-max.
 //                      Sampling (Sec. 2.1): test siblings in index order with u < min(1, r/q); the
@@ -128,8 +131,10 @@ __device__ __forceinline__ float load_logit(const void* base, int is_bf16, size_
 // without the rejected tokens (running sums in double, one contiguous run of tokens per thread).
 __device__ __noinline__ void deterministic_walk(const AcceptParams& p, int b) {
     __shared__ int s_par[HS_MAX_NODES], s_tok[HS_MAX_NODES], s_rej[HS_MAX_NODES];
+    __shared__ float s_pt[HS_MAX_NODES], s_u[HS_MAX_NODES];     // p(token of node j | its parent), its accept uniform
     __shared__ double s_scan[HS_ROW_THREADS / 32];
     __shared__ double s_phase[64];
+    __shared__ double s_wp[64][HS_ROW_THREADS / 32];     // per (phase, warp) sums of pass 1
     __shared__ int s_pick[2];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x;
     const int koff = p.pr.keep_off[b];
@@ -148,6 +153,22 @@ __device__ __noinline__ void deterministic_walk(const AcceptParams& p, int b) {
     __syncthreads();
     const float invT = LOG2E / p.temperature[b];
     const size_t esz = p.is_bf16 ? 2 : 4;
+    // every candidate's probability under its parent's target row and its uniform, all nodes at once (one round
+    // trip instead of one per sibling test); the walk below then runs from shared memory
+    for (int j = 1 + tid; j < nk; j += nthr) {
+        const int par = s_par[j];
+        const int orig = p.pr.keep_idx[koff + j];
+        float pt = 0.f;
+        if (par >= 0 && par < nk) {
+            const int prow_i = p.target_layout == HS_ROWS_ORIGINAL ? nbase + p.pr.keep_idx[koff + par] : koff + par;
+            const char* row = (const char*)p.target + (size_t)prow_i * p.row_stride * esz;
+            const float2 ms = __ldcg(&p.ro.tgt_ms[koff + par]);      // written by another CTA of this launch
+            pt = exp2f((fmaxf(load_logit(row, p.is_bf16, s_tok[j]), -1e30f) - ms.x) * invT) * (1.f / ms.y);
+        }
+        s_pt[j] = pt;
+        s_u[j] = p.uniforms ? p.uniforms[nbase + orig] : philox_uniform(p.seed, p.offset, b, orig, 0);
+    }
+    __syncthreads();
     int cur = 0, len = 0, bonus = -1;
     for (int step = 0; step < nk; ++step) {
         if (tid == 0 && len < cap) {
@@ -164,11 +185,9 @@ __device__ __noinline__ void deterministic_walk(const AcceptParams& p, int b) {
         for (int j = cur + 1; j < nk; ++j) {                     // siblings in index order (every thread the same)
             if (s_par[j] != cur) continue;
             const int t = s_tok[j];
-            const float pt = exp2f((fmaxf(load_logit(prow, p.is_bf16, t), -1e30f) - pm) * invT) * ips;
+            const float pt = s_pt[j];
             const float a = fminf(1.f, pt / (float)W);
-            const int orig = p.pr.keep_idx[koff + j];
-            const float u = p.uniforms ? p.uniforms[nbase + orig] : philox_uniform(p.seed, p.offset, b, orig, 0);
-            if (u < a) { accepted = j; break; }
+            if (s_u[j] < a) { accepted = j; break; }
             const double W_next = W - (double)pt;
             if (!(W_next > 0.0)) { nrej = 0; W = 1.0; break; }  // nothing left: fall back to p
             if (tid == 0) s_rej[nrej] = t;
@@ -190,7 +209,8 @@ __device__ __noinline__ void deterministic_walk(const AcceptParams& p, int b) {
         __syncthreads();                                         // s_rej, s_pick
         const int ve = p.is_bf16 ? 8 : 4;
         const int phase_vecs = nthr * 4;
-        const int nph = (p.nvec + phase_vecs - 1) / phase_vecs;  // <= 64 for vocabularies up to 2^19 bf16 (larger ones: status below)
+        // (at most 64 phases: the launcher refuses vocabularies of more than 32 chunks = 64 phases)
+        const int nph = min((p.nvec + phase_vecs - 1) / phase_vecs, 64);
         // masses of this thread's 4 vectors of phase ph (0 past the vocabulary and for rejected tokens)
         auto phase_mass = [&](int ph, float (&m)[4][8]) {
             uint4 d[4];
@@ -221,6 +241,7 @@ __device__ __noinline__ void deterministic_walk(const AcceptParams& p, int b) {
             }
         };
         int last_pos = -1;
+#pragma unroll 2
         for (int ph = 0; ph < nph; ++ph) {
             float m[4][8];
             phase_mass(ph, m);
@@ -233,15 +254,15 @@ __device__ __noinline__ void deterministic_walk(const AcceptParams& p, int b) {
                     if (m[q][e] > 0.f) last_pos = ((ph * phase_vecs + tid * 4 + q) * ve + e);
                 }
             const double w = warp_sum_d(mine);
-            if (lane == 0) s_scan[warp] = w;
-            __syncthreads();
-            if (tid == 0) {
-                double t = 0.0;
-                for (int w2 = 0; w2 < nthr / 32; ++w2) t += s_scan[w2];
-                s_phase[ph] = t;
-            }
-            __syncthreads();
+            if (lane == 0) s_wp[ph][warp] = w;           // (no barrier per phase: the loads of the next one go out)
         }
+        __syncthreads();
+        for (int ph = tid; ph < nph; ph += nthr) {
+            double t = 0.0;
+            for (int w2 = 0; w2 < nthr / 32; ++w2) t += s_wp[ph][w2];
+            s_phase[ph] = t;
+        }
+        __syncthreads();
         double total = 0.0;
         for (int ph = 0; ph < nph; ++ph) total += s_phase[ph];
         const double goal = (double)ufin * total;
