@@ -3,35 +3,30 @@
 // CTA = (block of 128 query rows, KV split, sequence x kv-head).  The GQA group times the kept tree
 // nodes forms the dense M dimension: query row r = node * G + g.  The KV prefix is cut into tiles of
 // 64 keys that are shared out evenly over the splits; a CTA requests its first tiles by TMA
-// (cp.async.bulk.tensor into 128-byte-swizzled shared memory, one mbarrier per stage, four stages)
-// before it waits for the kernel ahead of it in the stream, because the cache does not depend on the
-// pruned tree.  The <= 128 tree keys are gathered with plain loads (their rows may be indirect) and
-// belong to the last split.  S = Q K^T and O += P V run on the tensor cores with fp32 accumulation;
-// the softmax is the online (running max / running sum) form in base 2.  Prefix columns are fully
-// visible, tree column j is visible to row r iff bit j of the ancestor mask of r's node is set.
-// The splits of one (query block, head) form a thread-block cluster: every CTA leaves its partial
-// (max, sum, O) in its own shared memory and, after a cluster barrier, merges one slice of the rows
-// by reading the other CTAs' partials through distributed shared memory.  No partial ever goes to
-// global memory and there is no second launch.
-#include <cooperative_groups.h>
+// (cp.async.bulk.tensor into 128-byte-swizzled shared memory, four stages, K and V on mbarriers of
+// their own) before it waits for the kernel ahead of it in the stream, because the cache does not
+// depend on the pruned tree.  The <= 128 tree keys are gathered with plain loads (their rows may be
+// indirect) and belong to the last split.  S = Q K^T and O += P V run on the 5th-generation tensor
+// cores (tcgen05.mma, accumulators in tensor memory) with fp32 accumulation; the softmax is the
+// online (running max / running sum) form in base 2.  Prefix columns are fully visible, tree column j
+// is visible to row r iff bit j of the ancestor mask of r's node is set.  The splits of one (query
+// block, head) form a thread-block cluster: every CTA stages its partial (max, sum, O) in its own
+// shared memory and pushes each owner's rows there by bulk copies through distributed shared memory;
+// an owner merges its rows once all pieces have landed.  No partial ever goes to global memory and
+// there is no second launch.
 #include <math_constants.h>
 
 #include "hs_common.cuh"
 #include "hs_layout.h"
 #include "hs_ptx.cuh"
 
-namespace cg = cooperative_groups;
-
-#define ATT_THREADS 256
 #define ATT_BM 128
 #define ATT_BN 64
-#define ATT_STAGES 4
 #define ATT_MAX_SPLIT 8
 #define ATT_TILE_BYTES (ATT_BN * HS_HEAD_DIM * 2)   // 16 KiB: one K or V tile
 #define ATT_STAGE_BYTES (2 * ATT_TILE_BYTES)
 #define ATT_Q_BYTES (ATT_BM * HS_HEAD_DIM * 2)      // 32 KiB
 #define ATT_PO_STRIDE (HS_HEAD_DIM + 4)             // floats per row of the partial O (padding: bank spread)
-#define ATT_SMEM_BYTES (ATT_STAGES * ATT_STAGE_BYTES + ATT_Q_BYTES + 1024)
 #define LOG2E 1.4426950408889634f
 #define LN2 0.6931471805599453f
 
@@ -53,23 +48,6 @@ struct AttnParams {
     int* err;
 };
 
-// ---- PTX wrappers ------------------------------------------------------------------------------
-__device__ __forceinline__ void ldsm_x4(unsigned int addr, unsigned int& r0, unsigned int& r1, unsigned int& r2,
-                                        unsigned int& r3) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(unsigned int addr, unsigned int& r0, unsigned int& r1, unsigned int& r2,
-                                          unsigned int& r3) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float* c, const unsigned int* a, unsigned int b0, unsigned int b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
 __device__ __forceinline__ unsigned int pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<unsigned int*>(&v);
@@ -92,322 +70,8 @@ __device__ __forceinline__ void prefix_range(int L, int nsplit, int split, int& 
     t1 = min(t0 + per, t_prefix);
 }
 
-__global__ void __launch_bounds__(ATT_THREADS, 1)
-tree_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV) {
-    extern __shared__ unsigned char smem_raw[];
-    cg::cluster_group cluster = cg::this_cluster();
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int pair = blockIdx.z, b = pair / p.hkv, h = pair % p.hkv;
-    const int split = blockIdx.y;
-    const int m0 = blockIdx.x * ATT_BM;
-
-    const unsigned int smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    unsigned char* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    const unsigned int sQ = smem_base + ATT_STAGES * ATT_STAGE_BYTES;
-    const unsigned int bar0 = sQ + ATT_Q_BYTES;
-
-    // ---- before the dependency wait: barriers, and the first KV prefix tiles (inputs of the caller) ------
-    const int kv0 = p.kv_off[b];
-    const int L = p.kv_off[b + 1] - kv0;
-    int t_prefix, t0, t1;
-    prefix_range(L, p.nsplit, split, t_prefix, t0, t1);
-    const int np = t1 - t0;                          // prefix tiles of this CTA
-    auto issue_prefix = [&](int i) {                 // thread 0: tile i of this CTA into stage i % ATT_STAGES
-        const int stage = i % ATT_STAGES;
-        const unsigned int sK = smem_base + stage * ATT_STAGE_BYTES, sV = sK + ATT_TILE_BYTES;
-        const unsigned int bar = bar0 + stage * 8;
-        const int tok = kv0 + (t0 + i) * ATT_BN;
-        mbar_expect_tx(bar, ATT_STAGE_BYTES);
-        if (p.head_first) {      // tensor dims (d, token, head)
-            tma_load_3d(sK, &tmK, 0, tok, h, bar);
-            tma_load_3d(sK + ATT_TILE_BYTES / 2, &tmK, 64, tok, h, bar);
-            tma_load_3d(sV, &tmV, 0, tok, h, bar);
-            tma_load_3d(sV + ATT_TILE_BYTES / 2, &tmV, 64, tok, h, bar);
-        } else {                 // tensor dims (d, head, token)
-            tma_load_3d(sK, &tmK, 0, h, tok, bar);
-            tma_load_3d(sK + ATT_TILE_BYTES / 2, &tmK, 64, h, tok, bar);
-            tma_load_3d(sV, &tmV, 0, h, tok, bar);
-            tma_load_3d(sV + ATT_TILE_BYTES / 2, &tmV, 64, h, tok, bar);
-        }
-    };
-    const int pre = min(np, ATT_STAGES);
-    if (tid == 0) {
-        for (int i = 0; i < ATT_STAGES; ++i) mbar_init(bar0 + i * 8, 1);
-        mbar_init_fence();
-        for (int i = 0; i < pre; ++i) issue_prefix(i);
-    }
-    pdl_launch_dependents();
-    pdl_wait();                                      // the pruned tree, q, k_tree, v_tree come from upstream
-    __syncthreads();
-
-    const int nk = (p.status[b] == 0) ? p.n_keep[b] : 0;
-    const int M = nk * p.G;
-    if (m0 >= M) {                                   // nothing to do (the same for every CTA of the cluster)
-        for (int i = 0; i < pre; ++i) mbar_wait(bar0 + i * 8, 0u, p.err);   // no copy may outlive the CTA
-        return;
-    }
-    const int koff = p.keep_off[b];
-    const int nt_tree = (split == p.nsplit - 1) ? (nk + ATT_BN - 1) / ATT_BN : 0;
-    const int ntiles = np + nt_tree;
-
-    // tree keys/values: gathered rows, 16-byte loads, swizzled stores (2 x 1024 chunks / 256 threads)
-    auto gather_tree = [&](int i) {
-        unsigned char* gK = smem_gen + (i % ATT_STAGES) * ATT_STAGE_BYTES;
-        unsigned char* gV = gK + ATT_TILE_BYTES;
-        const int j0 = (i - np) * ATT_BN;
-        uint4 kvv[4], vvv[4];
-#pragma unroll
-        for (int it = 0; it < 4; ++it) {
-            const int c = tid + it * ATT_THREADS;       // 0..1023
-            const int j = j0 + (c >> 4);
-            kvv[it] = make_uint4(0, 0, 0, 0);
-            vvv[it] = make_uint4(0, 0, 0, 0);
-            if (j < nk) {
-                const int trow = (p.layout == HS_ROWS_ORIGINAL) ? p.node_off[b] + p.keep_idx[koff + j] : koff + j;
-                const size_t off = ((size_t)trow * p.hkv + h) * HS_HEAD_DIM + (c & 15) * 8;
-                kvv[it] = __ldg(reinterpret_cast<const uint4*>(p.k_tree + off));
-                vvv[it] = __ldg(reinterpret_cast<const uint4*>(p.v_tree + off));
-            }
-        }
-#pragma unroll
-        for (int it = 0; it < 4; ++it) {
-            const int c = tid + it * ATT_THREADS;
-            *reinterpret_cast<uint4*>(gK + tile_off(c >> 4, c & 15)) = kvv[it];
-            *reinterpret_cast<uint4*>(gV + tile_off(c >> 4, c & 15)) = vvv[it];
-        }
-    };
-
-    // ---- query tile -> shared memory (each warp its own 16 rows), ancestor masks, output rows ------------
-    const int gid = lane >> 2, qd = (lane & 3) * 2;
-    int my_orow = -1;                                // lanes 0..15: output row of query row warp*16 + lane
-    unsigned long long my_m0 = 0ull, my_m1 = 0ull;
-    if (lane < 16) {
-        const int r = m0 + warp * 16 + lane;
-        if (r < M) {
-            const int node = r / p.G, g = r - node * p.G;
-            const int trow = (p.layout == HS_ROWS_ORIGINAL) ? p.node_off[b] + p.keep_idx[koff + node] : koff + node;
-            my_orow = trow * p.hq + h * p.G + g;
-            my_m0 = p.anc_mask[2 * (size_t)(koff + node)];
-            my_m1 = p.anc_mask[2 * (size_t)(koff + node) + 1];
-        }
-    }
-    {
-        uint4 qv[8];
-#pragma unroll
-        for (int it = 0; it < 8; ++it) {
-            const int c = lane + 32 * it;                // 16 rows x 16 chunks
-            const int orow = __shfl_sync(HS_FULL_MASK, my_orow, c >> 4);
-            qv[it] = make_uint4(0, 0, 0, 0);
-            if (orow >= 0) qv[it] = __ldg(reinterpret_cast<const uint4*>(p.q + (size_t)orow * HS_HEAD_DIM) + (c & 15));
-        }
-#pragma unroll
-        for (int it = 0; it < 8; ++it) {
-            const int c = lane + 32 * it;
-            *reinterpret_cast<uint4*>(smem_gen + ATT_STAGES * ATT_STAGE_BYTES + q_off(warp * 16 + (c >> 4), c & 15)) = qv[it];
-        }
-    }
-    for (int i = np; i < min(ntiles, ATT_STAGES); ++i) gather_tree(i);     // tree tiles that open the pipeline
-    __syncthreads();
-    unsigned int qf[8][4];
-#pragma unroll
-    for (int ks = 0; ks < 8; ++ks)
-        ldsm_x4(sQ + q_off(warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, 2 * ks + (lane >> 4)),
-                qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
-    const int orow[2] = {__shfl_sync(HS_FULL_MASK, my_orow, gid), __shfl_sync(HS_FULL_MASK, my_orow, gid + 8)};
-    const unsigned long long mk[2][2] = {
-        {__shfl_sync(HS_FULL_MASK, my_m0, gid), __shfl_sync(HS_FULL_MASK, my_m1, gid)},
-        {__shfl_sync(HS_FULL_MASK, my_m0, gid + 8), __shfl_sync(HS_FULL_MASK, my_m1, gid + 8)}};
-
-    float oacc[16][4];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) { oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f; }
-    float mrun[2] = {-CUDART_INF_F, -CUDART_INF_F};
-    float lrun[2] = {0.f, 0.f};
-
-    // ---- KV tiles ------------------------------------------------------------------------------------------
-#pragma unroll 1
-    for (int i = 0; i < ntiles; ++i) {
-        const int stage = i % ATT_STAGES;
-        const bool is_tree = i >= np;
-        if (!is_tree) mbar_wait(bar0 + stage * 8, (unsigned int)(i / ATT_STAGES) & 1u, p.err);
-        const unsigned int sK = smem_base + stage * ATT_STAGE_BYTES, sV = sK + ATT_TILE_BYTES;
-
-        // S = Q K^T (16 x 64 per warp)
-        float sacc[8][4];
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-            sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f;
-            const int key = nt * 8 + (lane & 7);
-#pragma unroll
-            for (int kp = 0; kp < 4; ++kp) {
-                unsigned int b0, b1, b2, b3;
-                ldsm_x4(sK + tile_off(key, kp * 4 + (lane >> 3)), b0, b1, b2, b3);
-                mma_bf16(sacc[nt], qf[2 * kp], b0, b1);
-                mma_bf16(sacc[nt], qf[2 * kp + 1], b2, b3);
-            }
-        }
-        // scale, mask, online softmax
-        const int col0 = is_tree ? (i - np) * ATT_BN : (t0 + i) * ATT_BN;
-        const int limit = is_tree ? nk : L;
-        float mx[2] = {-CUDART_INF_F, -CUDART_INF_F};
-        // a tree tile of 64 keys lies inside one 64-bit word of the ancestor mask
-        const unsigned long long mw[2] = {col0 == 0 ? mk[0][0] : mk[0][1], col0 == 0 ? mk[1][0] : mk[1][1]};
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int cl = nt * 8 + qd + (e & 1);
-                const int x = e >> 1;
-                bool vis = col0 + cl < limit;
-                if (is_tree && vis) vis = (mw[x] >> cl) & 1ull;
-                const float sv = vis ? sacc[nt][e] * p.scale_log2 : -CUDART_INF_F;
-                sacc[nt][e] = sv;
-                mx[x] = fmaxf(mx[x], sv);
-            }
-        }
-        float corr[2], muse[2];
-#pragma unroll
-        for (int x = 0; x < 2; ++x) {
-            mx[x] = fmaxf(mx[x], __shfl_xor_sync(HS_FULL_MASK, mx[x], 1));
-            mx[x] = fmaxf(mx[x], __shfl_xor_sync(HS_FULL_MASK, mx[x], 2));
-            const float mnew = fmaxf(mrun[x], mx[x]);
-            muse[x] = (mnew == -CUDART_INF_F) ? 0.f : mnew;
-            corr[x] = ex2_approx(mrun[x] - muse[x]);
-            mrun[x] = mnew;
-            lrun[x] *= corr[x];
-        }
-#pragma unroll
-        for (int q = 0; q < 16; ++q) {
-            oacc[q][0] *= corr[0]; oacc[q][1] *= corr[0];
-            oacc[q][2] *= corr[1]; oacc[q][3] *= corr[1];
-        }
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float pv = ex2_approx(sacc[nt][e] - muse[e >> 1]);
-                sacc[nt][e] = pv;
-                lrun[e >> 1] += pv;
-            }
-        }
-        // O += P V
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-            unsigned int pa[4];
-            pa[0] = pack_bf16(sacc[2 * kk][0], sacc[2 * kk][1]);
-            pa[1] = pack_bf16(sacc[2 * kk][2], sacc[2 * kk][3]);
-            pa[2] = pack_bf16(sacc[2 * kk + 1][0], sacc[2 * kk + 1][1]);
-            pa[3] = pack_bf16(sacc[2 * kk + 1][2], sacc[2 * kk + 1][3]);
-            const int key = kk * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
-#pragma unroll
-            for (int dc = 0; dc < 8; ++dc) {
-                unsigned int b0, b1, b2, b3;
-                ldsm_x4_t(sV + tile_off(key, dc * 2 + (lane >> 4)), b0, b1, b2, b3);
-                mma_bf16(oacc[2 * dc], pa, b0, b1);
-                mma_bf16(oacc[2 * dc + 1], pa, b2, b3);
-            }
-        }
-        __syncthreads();     // every warp is done with the stage
-        const int nx = i + ATT_STAGES;
-        if (nx < ntiles) {
-            if (nx < np) { if (tid == 0) issue_prefix(nx); }
-            else gather_tree(nx);        // visible to all warps after the barrier that ends the next tile
-        }
-    }
-
-    // ---- epilogue ----------------------------------------------------------------------------------------------
-#pragma unroll
-    for (int x = 0; x < 2; ++x) {
-        lrun[x] += __shfl_xor_sync(HS_FULL_MASK, lrun[x], 1);
-        lrun[x] += __shfl_xor_sync(HS_FULL_MASK, lrun[x], 2);
-    }
-    if (p.nsplit == 1) {
-#pragma unroll
-        for (int x = 0; x < 2; ++x) {
-            if (orow[x] < 0) continue;
-            const float inv = lrun[x] > 0.f ? 1.f / lrun[x] : 0.f;
-            __nv_bfloat16* dst = p.out + (size_t)orow[x] * HS_HEAD_DIM;
-#pragma unroll
-            for (int q = 0; q < 16; ++q)
-                *reinterpret_cast<unsigned int*>(dst + q * 8 + qd) =
-                    pack_bf16(oacc[q][2 * x] * inv, oacc[q][2 * x + 1] * inv);
-            if (p.lse_out && (lane & 3) == 0) p.lse_out[orow[x]] = (mrun[x] + log2f(lrun[x])) * LN2;
-        }
-        return;
-    }
-
-    // ---- merge across the splits of the cluster through distributed shared memory --------------------------------
-    float* po = reinterpret_cast<float*>(smem_gen);                              // [128][ATT_PO_STRIDE]
-    float2* pml = reinterpret_cast<float2*>(smem_gen + ATT_BM * ATT_PO_STRIDE * 4);  // [128] {max (base 2), sum}
-#pragma unroll
-    for (int x = 0; x < 2; ++x) {
-        const int rl = warp * 16 + gid + 8 * x;
-#pragma unroll
-        for (int q = 0; q < 16; ++q)
-            *reinterpret_cast<float2*>(po + rl * ATT_PO_STRIDE + q * 8 + qd) = make_float2(oacc[q][2 * x], oacc[q][2 * x + 1]);
-        if ((lane & 3) == 0) pml[rl] = make_float2(mrun[x], lrun[x]);
-    }
-    cluster.sync();
-    {
-        const int ns = p.nsplit;                         // 2, 4 or 8
-        const int rows_per = ATT_BM / ns;                // rows this CTA merges
-        const int tpr = ATT_THREADS / rows_per;          // threads per row
-        const int rl = split * rows_per + tid / tpr;     // row inside the query block
-        const int c0 = (tid % tpr) * (HS_HEAD_DIM / tpr);    // first of this thread's HS_HEAD_DIM / tpr columns
-        const int nch = HS_HEAD_DIM / tpr / 4;           // float4 chunks per thread: ns * nch = 16
-        float2 ml[ATT_MAX_SPLIT];
-        float Mx = -CUDART_INF_F;
-#pragma unroll
-        for (int s = 0; s < ATT_MAX_SPLIT; ++s) {
-            ml[s] = make_float2(-CUDART_INF_F, 0.f);
-            if (s < ns) ml[s] = cluster.map_shared_rank(pml, s)[rl];
-            Mx = fmaxf(Mx, ml[s].x);
-        }
-        float w[ATT_MAX_SPLIT], lsum = 0.f;
-#pragma unroll
-        for (int s = 0; s < ATT_MAX_SPLIT; ++s) {
-            w[s] = (ml[s].x == -CUDART_INF_F) ? 0.f : ex2_approx(ml[s].x - Mx);
-            lsum = fmaf(w[s], ml[s].y, lsum);
-        }
-        const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
-        const int r = m0 + rl;
-        if (r < M) {
-            const int node = r / p.G, g = r - node * p.G;
-            const int trow = (p.layout == HS_ROWS_ORIGINAL) ? p.node_off[b] + p.keep_idx[koff + node] : koff + node;
-            const size_t orow_g = (size_t)trow * p.hq + h * p.G + g;
-            // the thread's 16 remote float4 (ns partials x nch chunks) are requested together
-            float4 v[16];
-#pragma unroll
-            for (int k = 0; k < 16; ++k) {
-                const int s = k % ns, ch = k / ns;
-                v[k] = *reinterpret_cast<const float4*>(cluster.map_shared_rank(po, s) + rl * ATT_PO_STRIDE + c0 + ch * 4);
-            }
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int k = 0; k < 16; ++k) {
-                const int s = k % ns, ch = k / ns;
-                float ws = w[0];
-#pragma unroll
-                for (int q = 1; q < ATT_MAX_SPLIT; ++q) ws = (s == q) ? w[q] : ws;
-                acc.x = fmaf(ws, v[k].x, acc.x); acc.y = fmaf(ws, v[k].y, acc.y);
-                acc.z = fmaf(ws, v[k].z, acc.z); acc.w = fmaf(ws, v[k].w, acc.w);
-                if (s == ns - 1) {
-                    uint2 packed;
-                    packed.x = pack_bf16(acc.x * inv, acc.y * inv);
-                    packed.y = pack_bf16(acc.z * inv, acc.w * inv);
-                    *reinterpret_cast<uint2*>(p.out + orow_g * HS_HEAD_DIM + c0 + ch * 4) = packed;
-                    acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-            }
-            if (p.lse_out && (tid % tpr) == 0) p.lse_out[orow_g] = (Mx + log2f(lsum)) * LN2;
-        }
-    }
-    cluster.sync();      // nobody leaves while its shared memory may still be read
-}
-
-
 // =====================================================================================================
-// tcgen05 version: S = Q K^T and O += P V by the 5th-generation tensor cores, accumulators in tensor
+// The kernel: S = Q K^T and O += P V by the 5th-generation tensor cores, accumulators in tensor
 // memory.  Two softmax warpgroups run two independent online-softmax streams over the block's 128 query
 // rows: warpgroup g takes the KV tiles i = g, g + 2, ... and keeps its own S buffer, P buffer, running
 // (max, sum) and O accumulator; thread t of a warpgroup owns query row t (= tensor-memory lane t), so the
@@ -432,8 +96,7 @@ tree_attn_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, co
 __global__ void __launch_bounds__(UM_THREADS, 1)
 tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV) {
     extern __shared__ unsigned char smem_raw[];
-    cg::cluster_group cluster = cg::this_cluster();
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, warp = tid >> 5;
     const int pair = blockIdx.z, b = pair / p.hkv, h = pair % p.hkv;
     const int split = blockIdx.y;
     const int m0 = blockIdx.x * ATT_BM;
@@ -944,10 +607,10 @@ static bool make_kv_map(hs_ctx* ctx, CUtensorMap* tm, const void* base, const hs
 // KV splits (= cluster size): the one with the fewest tile steps on the critical path, waves of CTAs (as
 // many clusters of that size as the device runs at once) times tiles per CTA.  `step` = 1 tries 1..8,
 // `step` = 2 only powers of two.
-static int choose_splits(int base_ctas, int sm_count, int prefix_tiles, const int* cluster_cap, bool pow2) {
+static int choose_splits(int base_ctas, int sm_count, int prefix_tiles, const int* cluster_cap) {
     int best = 1;
     long best_cost = 0;
-    for (int s = 1; s <= ATT_MAX_SPLIT; s = pow2 ? s * 2 : s + 1) {
+    for (int s = 1; s <= ATT_MAX_SPLIT; ++s) {
         if (s > 1 && s > prefix_tiles) break;
         const long ctas = (long)base_ctas * s;
         const long cap = cluster_cap[s] > 0 ? cluster_cap[s] : sm_count;
@@ -980,17 +643,11 @@ hs_status hs_launch_attention(hs_ctx* ctx, const hs_pruned_tree* pruned, const h
                               const void* k_tree, const void* v_tree, const void* k_cache, const void* v_cache,
                               void* out, float* lse_out, cudaStream_t stream) {
     static bool attr_set = false;
-    static bool legacy = false;                    // HS_ATTN_MMA_SYNC=1: the mma.sync kernel instead of tcgen05
-    static int cap_umma[ATT_MAX_SPLIT + 1], cap_legacy[ATT_MAX_SPLIT + 1];   // CTAs that run at once in clusters of s
+    static int cap_umma[ATT_MAX_SPLIT + 1];          // CTAs that run at once in clusters of s
     if (!attr_set) {
-        const char* e = getenv("HS_ATTN_MMA_SYNC");
-        legacy = e && e[0] == '1';
-        if (cudaFuncSetAttribute(tree_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES) !=
-                cudaSuccess ||
-            cudaFuncSetAttribute(tree_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, UM_SMEM_BYTES) !=
-                cudaSuccess)
+        if (cudaFuncSetAttribute(tree_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, UM_SMEM_BYTES) !=
+            cudaSuccess)
             return HS_ERR_CUDA;
-        query_cluster_caps(tree_attn_kernel, ATT_THREADS, ATT_SMEM_BYTES, ctx->sm_count, cap_legacy);
         query_cluster_caps(tree_attn_umma_kernel, UM_THREADS, UM_SMEM_BYTES, ctx->sm_count, cap_umma);
         attr_set = true;
     }
@@ -1018,8 +675,7 @@ hs_status hs_launch_attention(hs_ctx* ctx, const hs_pruned_tree* pruned, const h
     const int pairs = d->batch * d->hkv;
     const int mblocks = (p.G * d->max_nodes + ATT_BM - 1) / ATT_BM;
     const int prefix_tiles = (d->max_kv_len + ATT_BN - 1) / ATT_BN;
-    p.nsplit = legacy ? choose_splits(pairs * mblocks, ctx->sm_count, prefix_tiles, cap_legacy, true)
-                      : choose_splits(pairs * mblocks, ctx->sm_count, prefix_tiles, cap_umma, false);
+    p.nsplit = choose_splits(pairs * mblocks, ctx->sm_count, prefix_tiles, cap_umma);
 
     CUtensorMap tmK, tmV;
     memset(&tmK, 0, sizeof(tmK));
@@ -1029,8 +685,6 @@ hs_status hs_launch_attention(hs_ctx* ctx, const hs_pruned_tree* pruned, const h
             return HS_ERR_CUDA;
     }
     const dim3 grid(mblocks, p.nsplit, pairs), cl(1, p.nsplit, 1);
-    cudaError_t e = legacy
-        ? hs_launch(tree_attn_kernel, grid, dim3(ATT_THREADS), ATT_SMEM_BYTES, stream, ctx->pdl, cl, p, tmK, tmV)
-        : hs_launch(tree_attn_umma_kernel, grid, dim3(UM_THREADS), UM_SMEM_BYTES, stream, ctx->pdl, cl, p, tmK, tmV);
+    cudaError_t e = hs_launch(tree_attn_umma_kernel, grid, dim3(UM_THREADS), UM_SMEM_BYTES, stream, ctx->pdl, cl, p, tmK, tmV);
     return e == cudaSuccess ? HS_OK : HS_ERR_CUDA;
 }
