@@ -172,8 +172,9 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, MODE ? 4 : 2) quantify_kernel(
     };
     // ---- maxima ---------------------------------------------------------------------------
     // Rolled loops over the vectors need 40 registers instead of 64, so six CTAs share an SM: measured 20 % faster
-    // on launches of many waves, 3 us slower on a launch that is resident at once (the launcher chooses).
-    constexpr int UJ = MODE == 2 ? 2 : VPT, UC = MODE == 2 ? 1 : VPT;
+    // on launches of many waves, 3 us slower on a launch that is resident at once (the launcher chooses).  The
+    // candidate scan is rolled in both staged variants: few threads run it, mostly from a cold instruction cache.
+    constexpr int UJ = MODE == 2 ? 2 : VPT, UC = MODE != 0 ? 1 : VPT;
     float vmax[STAGED ? 1 : VPT];
     float tmax = -CUDART_INF_F;
 #pragma unroll UJ
