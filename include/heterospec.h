@@ -23,7 +23,13 @@
  *     The small descriptor structs (hs_tree_batch, hs_policy, ...) are host structs read during
  *     the call.  The library owns only the workspace created by hs_create.
  *   - All four step calls enqueue work on the caller's stream and return without synchronising.
- *     `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     `stream` is a cudaStream_t passed as void* (NULL = default stream).  A context serves one
+ *     stream at a time (its workspace is shared by the calls); the device of the context must be
+ *     the current device of the calling thread, otherwise the call returns HS_ERR_INVALID_ARG.
+ *   - Kernels are launched with programmatic stream serialisation: their prologue may overlap the
+ *     tail of the kernel ahead of them in the stream.  By default every read of caller memory comes
+ *     after the dependency wait, so inputs written by the preceding kernel (the draft model's LM
+ *     head, a cache append) are always complete.  hs_set_prefetch relaxes this per input class.
  *   - Errors: a bad argument or shape returns a non-zero hs_status and launches nothing.
  *     Data-dependent problems (malformed tree, token out of range) set status[b] != 0 on the
  *     device; later steps skip such a sequence (n_keep = 0, accept_len = 0).  Kernels never trap.
@@ -79,9 +85,24 @@ size_t hs_workspace_bytes(int32_t max_batch, int32_t max_rows, int32_t vocab, in
 hs_status hs_create(hs_ctx** ctx, int32_t device, size_t workspace_bytes);
 hs_status hs_destroy(hs_ctx* ctx);
 
+/* Inputs a kernel may start to fetch BEFORE it waits for the kernel ahead of it in the stream (see
+ * "Conventions").  Set a bit only if that input is complete before the call is enqueued, i.e. it is
+ * not written by the immediately preceding kernel of the stream: typically true for the KV cache
+ * prefix (appended a step earlier), true for logits only if something else separates producer and
+ * call.  Default 0: nothing is read early. */
+#define HS_PREFETCH_LOGITS 1   /* draft logits of hs_entropy_quantify */
+#define HS_PREFETCH_KV 2       /* k_cache / v_cache of hs_tree_verify_attention */
+hs_status hs_set_prefetch(hs_ctx* ctx, int32_t flags);
+
 /* Reads and clears the context's sticky device error word into *host_out (host pointer): HS_OK, or
  * HS_ERR_TIMEOUT if a kernel gave up a bounded wait since the last call.  Synchronises the device. */
 hs_status hs_device_error(hs_ctx* ctx, int32_t* host_out);
+
+/* Self-test of the bounded device-side wait (no counterpart in the paper): one thread waits on a
+ * barrier that nothing completes, gives up after `limit_ns` nanoseconds (clamped to 1 us .. 10 ms)
+ * and records HS_ERR_TIMEOUT in the context's error word, which hs_device_error then returns.  The
+ * kernel always terminates; the context stays usable. */
+hs_status hs_selftest_wait_timeout(hs_ctx* ctx, uint64_t limit_ns, hs_stream stream);
 
 /* ---- descriptors -------------------------------------------------------------------------- */
 
@@ -214,8 +235,13 @@ hs_status hs_tree_verify_attention(hs_ctx* ctx, const hs_pruned_tree* pruned, co
  * are read only by sequences in rejection mode; a caller without such sequences passes NULL (a
  * rejection-mode sequence then gets status HS_ERR_INVALID_ARG) and saves a launch.  mode[b]: hs_accept_mode;
  * temperature[b] > 0 for the two sampling modes, applied to both models.  Uniforms: Philox4x32-10 with key = seed, counter =
- * (offset, b, original node id, stream) with stream 0 = accept test of that node, 1 = final draw
- * (node 0); u = (x0 >> 8) * 2^-24.  If `uniforms` is not NULL it overrides the generator:
+ * (low word of offset, b, original node id, stream + 2 * (high word of offset)) with stream 0 = accept test of
+ * that node, 1 = final draw (node 0); offset < 2^63; u = (x0 >> 8) * 2^-24.
+ * Sibling candidates that carry the same token: the first in index order is the candidate, a later one
+ * is tested against the residual like any other (greedy: the lowest index is taken).
+ * path_cap: slots per sequence in path_*; a path longer than path_cap - 1 tokens is still walked and
+ * accept_len reports its true length, only the first path_cap entries are stored.
+ * If `uniforms` is not NULL it overrides the generator:
  * uniforms[node_off[b] + node] for accept tests and uniforms[n_nodes_total + b] for the final draw. */
 hs_status hs_accept_path(hs_ctx* ctx, const hs_tree_batch* tree, const hs_pruned_tree* pruned,
                          const void* target_logits, int32_t target_layout, const void* draft_logits,

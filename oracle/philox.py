@@ -4,9 +4,10 @@ Own implementation of the published algorithm (Salmon, Moraes, Dror, Shaw:
 "Parallel random numbers: as easy as 1, 2, 3", SC'11): ten rounds of two
 32x32->64 multiplications with the key bumped by the Weyl constants between
 rounds.  The verification path draws its uniforms as
-    u = (x0 >> 8) * 2^-24,   x = Philox(key = seed, counter = (offset, b, node, stream))
+    u = (x0 >> 8) * 2^-24,   x = Philox(key = seed, counter = (offset low word, b, node,
+                                                               stream + 2 * offset high word))
 with stream 0 for the accept test of ``node`` and stream 1 for the final
-(bonus-token) draw of sequence b (node = 0).
+(bonus-token) draw of sequence b (node = 0); offset < 2^63.
 """
 
 import numpy as np
@@ -33,5 +34,5 @@ def philox4x32_10(counter, key):
 def uniform(seed, offset, b, node, stream):
     """One uniform in [0, 1) with 24 random bits, as drawn by the acceptance step."""
     key = (int(seed) & _MASK, (int(seed) >> 32) & _MASK)
-    x = philox4x32_10((int(offset) & _MASK, int(b), int(node), int(stream)), key)
+    x = philox4x32_10((int(offset) & _MASK, int(b), int(node), int(stream) + 2 * (int(offset) >> 32)), key)
     return float(x[0] >> 8) * 2.0 ** -24

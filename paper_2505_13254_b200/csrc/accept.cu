@@ -40,7 +40,7 @@ struct AcceptParams {
     const void* draft;
     int64_t row_stride;
     int vocab, nvec, chunks, chunk_vecs, is_bf16, have_draft;
-    int batch, n_nodes_total, target_layout;
+    int batch, n_nodes_total, target_layout, part_rows;
     const int* node_off;
     const int* token;
     hs_pruned_tree pr;
@@ -185,12 +185,16 @@ __device__ __noinline__ void deterministic_walk(const AcceptParams& p, int b) {
         for (int j = cur + 1; j < nk; ++j) {                     // siblings in index order (every thread the same)
             if (s_par[j] != cur) continue;
             const int t = s_tok[j];
-            const float pt = s_pt[j];
+            float pt = s_pt[j];
+            for (int k = 0; k < nrej; ++k)                       // a token rejected at this node has left the residual
+                if (s_rej[k] == t) pt = 0.f;
             const float a = fminf(1.f, pt / (float)W);
             if (s_u[j] < a) { accepted = j; break; }
             const double W_next = W - (double)pt;
             if (!(W_next > 0.0)) { nrej = 0; W = 1.0; break; }  // nothing left: fall back to p
+            __syncthreads();                                     // (every thread walks the same way)
             if (tid == 0) s_rej[nrej] = t;
+            __syncthreads();
             ++nrej;
             W = W_next;
         }
@@ -422,7 +426,7 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 4) accept_rows_kernel(const __
             for (int w = 0; w < 8; ++w)
                 S += (s_w[w][0] == -CUDART_INF_F) ? 0.f : s_w[w][1] * ex2a((s_w[w][0] - M) * invT);
         }
-        p.partials[((size_t)which * HS_MAX_ROWS + k) * p.chunks + chunk] =
+        p.partials[((size_t)which * p.part_rows + k) * p.chunks + chunk] =
             make_uint4((unsigned int)best, (unsigned int)(best >> 32), __float_as_uint(M), __float_as_uint(S));
         __threadfence();
         int* cnt = &p.row_cnt[which * HS_MAX_ROWS + k];
@@ -437,7 +441,7 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 4) accept_rows_kernel(const __
     unsigned long long ck = 0ull;
     float cm = -CUDART_INF_F, cs = 0.f;
     if (lane < p.chunks) {
-        uint4 q = __ldcg(&p.partials[((size_t)which * HS_MAX_ROWS + k) * p.chunks + lane]);
+        uint4 q = __ldcg(&p.partials[((size_t)which * p.part_rows + k) * p.chunks + lane]);
         ck = ((unsigned long long)q.y << 32) | q.x;
         cm = __uint_as_float(q.z);
         cs = __uint_as_float(q.w);
@@ -458,10 +462,18 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 4) accept_rows_kernel(const __
     }
     }
     // ---- greedy sequences finish here: the last target row of a sequence to be merged walks its tree ------
-    if (md == HS_ACCEPT_REJECTION && !p.have_draft && which == 0 && i == 0 && tid == 0) {
+    if (md == HS_ACCEPT_REJECTION && !p.have_draft && which == 0 && i == 0) {
         // rejection sampling needs the draft distribution: the caller passed none
-        p.out.accept_len[b] = 0; p.out.bonus_token[b] = -1; p.out.terminal_rank[b] = -1;
-        p.out.status[b] = HS_ERR_INVALID_ARG;
+        const int cap = p.out.path_cap;
+        for (int j = tid; j < cap; j += HS_ROW_THREADS) {
+            p.out.path_nodes[b * cap + j] = -1;
+            p.out.path_compact[b * cap + j] = -1;
+            p.out.path_tokens[b * cap + j] = -1;
+        }
+        if (tid == 0) {
+            p.out.accept_len[b] = 0; p.out.bonus_token[b] = -1; p.out.terminal_rank[b] = -1;
+            p.out.status[b] = HS_ERR_INVALID_ARG;
+        }
     }
     if (which != 0 || md == HS_ACCEPT_REJECTION) return;
     __syncthreads();
@@ -793,7 +805,8 @@ hs_status hs_launch_accept(hs_ctx* ctx, const hs_tree_batch* tree, const hs_prun
     p.ro.tgt_ms = (float2*)(ctx->scratch + o); o += hs_align_up((size_t)rows * sizeof(float2), 256);
     p.ro.drf_ms = (float2*)(ctx->scratch + o); o += hs_align_up((size_t)rows * sizeof(float2), 256);
     p.partials = (uint4*)(ctx->scratch + o);
-    o += (size_t)(HS_MAX_ROWS + rows) * p.chunks * sizeof(uint4);
+    p.part_rows = rows;
+    o += (size_t)2 * rows * p.chunks * sizeof(uint4);
     if (o > ctx->scratch_bytes) return HS_ERR_WORKSPACE;
     p.row_cnt = ctx->counters + HS_CNT_ACC_ROW;
     p.seq_cnt = ctx->counters + HS_CNT_ACC_SEQ;
@@ -811,14 +824,11 @@ hs_status hs_launch_accept(hs_ctx* ctx, const hs_tree_batch* tree, const hs_prun
     const size_t walk_smem = 2 * (size_t)((p.nvec + WALK_CLUSTER - 1) / WALK_CLUSTER) * 16;
     p.staged = ((uintptr_t)p.target % 16 == 0) && ((uintptr_t)p.draft % 16 == 0) && ((size_t)row_stride * esz % 16 == 0) &&
                walk_smem <= 160 * 1024;
-    static bool walk_attr[64];               // per device: the kernel may use more than 48 KiB of shared memory
-    if (ctx->device >= 0 && ctx->device < 64 && !walk_attr[ctx->device]) {
+    if (!ctx->walk_ready) {                  // per device (= per context): more than 48 KiB of shared memory, 16-CTA clusters
         if (cudaFuncSetAttribute(accept_walk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024) != cudaSuccess ||
             cudaFuncSetAttribute(accept_walk_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
             return HS_ERR_CUDA;
-        walk_attr[ctx->device] = true;
-    } else if (ctx->device < 0 || ctx->device >= 64) {
-        p.staged = 0;
+        ctx->walk_ready = true;
     }
     e = hs_launch(accept_walk_kernel, dim3(p.batch * WALK_CLUSTER), dim3(WALK_THREADS), p.staged ? walk_smem : 0, stream,
                   ctx->pdl, dim3(1, 1, 1), p);

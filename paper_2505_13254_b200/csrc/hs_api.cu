@@ -5,6 +5,7 @@
 
 #include "hs_common.cuh"
 #include "hs_layout.h"
+#include "hs_ptx.cuh"
 
 extern "C" const char* hs_status_string(hs_status s) {
     switch (s) {
@@ -24,14 +25,14 @@ extern "C" const char* hs_status_string(hs_status s) {
 extern "C" size_t hs_workspace_bytes(int32_t max_batch, int32_t max_rows, int32_t vocab, int32_t hq, int32_t hkv) {
     if (max_batch < 1 || max_rows < 1 || vocab < 1 || hq < 1 || hkv < 1) return 0;
     size_t chunks = hs_row_chunks(vocab, HS_F32);
-    size_t quant = (size_t)max_rows * chunks * HS_ROW_PARTIAL_BYTES;
-    size_t accept = (size_t)max_rows * 2 * chunks * HS_ACC_PARTIAL_BYTES + (size_t)max_rows * 2 * 16;
-    // attention: room for HS_ATTN_WS_SPLITS partial (O, m, l) sets of every (row, head), floor 64 MiB
-    size_t attn = (size_t)max_rows * hq * (HS_HEAD_DIM + 2) * sizeof(float) * HS_ATTN_WS_SPLITS;
-    if (attn < ((size_t)64 << 20)) attn = (size_t)64 << 20;
+    // entropy pass: two partials per CTA, at most one CTA per SM (room for 1024)
+    size_t quant = (size_t)2 * 1024 * HS_ROW_PARTIAL_BYTES + 256;
+    // acceptance: three per-row result arrays (256-byte aligned each) + chunk partials of target and draft rows
+    size_t accept = 3 * hs_align_up((size_t)max_rows * 8, 256) +
+                    (size_t)2 * max_rows * chunks * HS_ACC_PARTIAL_BYTES;
+    // (the attention merges its KV splits on chip: no workspace)
     size_t scratch = quant > accept ? quant : accept;
-    if (attn > scratch) scratch = attn;
-    return HS_COUNTER_BYTES + hs_align_up(scratch, 256);
+    return HS_COUNTER_BYTES + hs_align_up(scratch, 256) + 256;
 }
 
 extern "C" hs_status hs_create(hs_ctx** out, int32_t device, size_t workspace_bytes) {
@@ -42,13 +43,14 @@ extern "C" hs_status hs_create(hs_ctx** out, int32_t device, size_t workspace_by
     HS_CUDA_OK(cudaGetDeviceCount(&ndev));
     if (device < 0 || device >= ndev) return HS_ERR_INVALID_ARG;
     HS_CUDA_OK(cudaSetDevice(device));
+    int sm_count = 0, major = 0;
+    HS_CUDA_OK(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, device));
+    HS_CUDA_OK(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device));
+    if (major != 10) return HS_ERR_UNSUPPORTED;                   // built for sm_100a only
     hs_ctx* c = new (std::nothrow) hs_ctx();
     if (!c) return HS_ERR_INVALID_ARG;
     c->device = device;
-    HS_CUDA_OK(cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device));
-    int major = 0;
-    HS_CUDA_OK(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device));
-    if (major != 10) { delete c; return HS_ERR_UNSUPPORTED; }     // built for sm_100a only
+    c->sm_count = sm_count;
     void* p = nullptr;
     if (cudaMalloc(&p, workspace_bytes) != cudaSuccess) { delete c; return HS_ERR_CUDA; }
     c->ws = (char*)p;
@@ -67,7 +69,11 @@ extern "C" hs_status hs_create(hs_ctx** out, int32_t device, size_t workspace_by
     c->encode_tiled = fn;
     const char* no_pdl = getenv("HS_DISABLE_PDL");
     c->pdl = !(no_pdl && no_pdl[0] == '1');
-    HS_CUDA_OK(cudaDeviceSynchronize());
+    c->prefetch = 0;
+    c->attn_ready = false;
+    c->walk_ready = false;
+    c->quant_ready = false;
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaFree(p); delete c; return HS_ERR_CUDA; }
     *out = c;
     return HS_OK;
 }
@@ -78,6 +84,34 @@ extern "C" hs_status hs_destroy(hs_ctx* ctx) {
     cudaFree(ctx->ws);
     delete ctx;
     return HS_OK;
+}
+
+// One thread waits on a barrier that nothing ever completes; the bounded wait gives up after limit_ns and
+// records HS_ERR_TIMEOUT in the context's error word.
+__global__ void wait_selftest_kernel(int* err, unsigned long long limit_ns) {
+    __shared__ unsigned long long s_bar;
+    const unsigned int bar = smem_u32(&s_bar);
+    mbar_init(bar, 1);
+    mbar_init_fence();
+    mbar_wait_limit(bar, 0u, err, limit_ns);
+}
+
+hs_status hs_launch_wait_selftest(hs_ctx* ctx, uint64_t limit_ns, cudaStream_t stream) {
+    wait_selftest_kernel<<<1, 1, 0, stream>>>(ctx->counters + HS_CNT_ERROR, (unsigned long long)limit_ns);
+    return cudaGetLastError() == cudaSuccess ? HS_OK : HS_ERR_CUDA;
+}
+
+extern "C" hs_status hs_set_prefetch(hs_ctx* ctx, int32_t flags) {
+    if (!ctx || (flags & ~(HS_PREFETCH_LOGITS | HS_PREFETCH_KV))) return HS_ERR_INVALID_ARG;
+    ctx->prefetch = flags;
+    return HS_OK;
+}
+
+extern "C" hs_status hs_selftest_wait_timeout(hs_ctx* ctx, uint64_t limit_ns, hs_stream stream) {
+    if (!ctx || !hs_on_device(ctx)) return HS_ERR_INVALID_ARG;
+    if (limit_ns < 1000ull) limit_ns = 1000ull;
+    if (limit_ns > 10000000ull) limit_ns = 10000000ull;
+    return hs_launch_wait_selftest(ctx, limit_ns, (cudaStream_t)stream);
 }
 
 extern "C" hs_status hs_device_error(hs_ctx* ctx, int32_t* host_out) {
@@ -114,7 +148,7 @@ static bool logits_ok(const void* p, hs_dtype dtype, int64_t row_stride, int32_t
 extern "C" hs_status hs_entropy_quantify(hs_ctx* ctx, const hs_tree_batch* tree, const void* draft_logits,
                                          hs_dtype dtype, int64_t row_stride, int32_t vocab,
                                          const hs_policy* policy, const hs_quant_out* out, hs_stream stream) {
-    if (!ctx || !out) return HS_ERR_INVALID_ARG;
+    if (!ctx || !out || !hs_on_device(ctx)) return HS_ERR_INVALID_ARG;
     if (!tree_ok(tree) || !policy_ok(policy) || !logits_ok(draft_logits, dtype, row_stride, vocab))
         return HS_ERR_INVALID_ARG;
     if (!out->row_max || !out->row_lse || !out->h_full || !out->i_topk || !out->i_trunc || !out->topk_val ||
@@ -126,7 +160,7 @@ extern "C" hs_status hs_entropy_quantify(hs_ctx* ctx, const hs_tree_batch* tree,
 
 extern "C" hs_status hs_stratify_prune(hs_ctx* ctx, const hs_tree_batch* tree, const hs_quant_out* quant,
                                        const hs_policy* policy, const hs_pruned_tree* out, hs_stream stream) {
-    if (!ctx || !quant || !out) return HS_ERR_INVALID_ARG;
+    if (!ctx || !quant || !out || !hs_on_device(ctx)) return HS_ERR_INVALID_ARG;
     if (!tree_ok(tree) || !policy_ok(policy)) return HS_ERR_INVALID_ARG;
     if (!quant->score || !quant->phi_star || !quant->depth || !quant->status) return HS_ERR_INVALID_ARG;
     if (!out->bin || !out->d_prime || !out->n_prime || !out->n_keep || !out->keep_off || !out->keep_idx ||
@@ -144,7 +178,8 @@ extern "C" hs_status hs_tree_verify_attention(hs_ctx* ctx, const hs_pruned_tree*
                                               const void* q, const void* k_tree, const void* v_tree,
                                               const void* k_cache, const void* v_cache, void* out,
                                               float* lse_out, hs_stream stream) {
-    if (!ctx || !d || !pruned_ok(pruned) || !q || !k_tree || !v_tree || !out) return HS_ERR_INVALID_ARG;
+    if (!ctx || !d || !pruned_ok(pruned) || !q || !k_tree || !v_tree || !out || !hs_on_device(ctx))
+        return HS_ERR_INVALID_ARG;
     if (d->batch < 1 || d->batch > HS_MAX_BATCH || d->max_rows < 1 || d->max_rows > HS_MAX_ROWS ||
         d->max_nodes < 1 || d->max_nodes > HS_MAX_NODES || d->kv_total < 0 || d->max_kv_len < 0 ||
         d->max_kv_len > d->kv_total || !d->kv_off)
@@ -169,7 +204,7 @@ extern "C" hs_status hs_accept_path(hs_ctx* ctx, const hs_tree_batch* tree, cons
                                     hs_dtype dtype, int64_t row_stride, int32_t vocab, const int32_t* mode,
                                     const float* temperature, uint64_t seed, uint64_t offset,
                                     const float* uniforms, const hs_accept_out* out, hs_stream stream) {
-    if (!ctx || !out || !mode || !temperature) return HS_ERR_INVALID_ARG;
+    if (!ctx || !out || !mode || !temperature || !hs_on_device(ctx) || (offset >> 63)) return HS_ERR_INVALID_ARG;
     if (!tree_ok(tree) || !pruned_ok(pruned) || !logits_ok(target_logits, dtype, row_stride, vocab))
         return HS_ERR_INVALID_ARG;
     if (draft_logits && ((uintptr_t)draft_logits & 15)) return HS_ERR_INVALID_ARG;
@@ -184,7 +219,8 @@ extern "C" hs_status hs_accept_path(hs_ctx* ctx, const hs_tree_batch* tree, cons
 extern "C" hs_status hs_philox_uniforms(hs_ctx* ctx, uint64_t seed, uint64_t offset, const int32_t* b,
                                         const int32_t* node, const int32_t* stream_id, int32_t count,
                                         float* out, hs_stream stream) {
-    if (!ctx || !b || !node || !stream_id || !out || count < 0) return HS_ERR_INVALID_ARG;
+    if (!ctx || !b || !node || !stream_id || !out || count < 0 || !hs_on_device(ctx) || (offset >> 63))
+        return HS_ERR_INVALID_ARG;
     if (count == 0) return HS_OK;
     return hs_launch_philox(seed, offset, b, node, stream_id, count, out, (cudaStream_t)stream);
 }

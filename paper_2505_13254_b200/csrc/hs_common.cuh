@@ -25,7 +25,18 @@ struct hs_ctx {
     size_t scratch_bytes;
     void* encode_tiled; // cuTensorMapEncodeTiled entry point
     bool pdl;           // launch kernels with programmatic stream serialisation
+    int prefetch;       // HS_PREFETCH_* bits: inputs a kernel may fetch before its dependency wait
+    bool attn_ready;    // attention kernel attributes set and cluster capacities queried on this device
+    int attn_cap[9];    // CTAs of the attention kernel that run at once in clusters of s = 1..8
+    bool walk_ready;    // acceptance walk kernel attributes set on this device
+    bool quant_ready;   // streaming entropy kernel: shared-memory attribute set on this device
 };
+
+// The context's device must be the calling thread's current device (launches go to the current device).
+static inline bool hs_on_device(const hs_ctx* ctx) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == ctx->device;
+}
 
 // Kernel launch with optional programmatic-dependent-launch attribute and thread-block cluster shape.
 template <typename... KArgs, typename... Args>
@@ -134,8 +145,10 @@ __device__ __forceinline__ unsigned int philox4x32_10_x0(unsigned int c0, unsign
 }
 __device__ __forceinline__ float philox_uniform(unsigned long long seed, unsigned long long offset, int b,
                                                 int node, int stream_id) {
+    // counter = (offset low word, b, node, stream + 2 * offset high word), key = seed
     unsigned int x0 = philox4x32_10_x0((unsigned int)offset, (unsigned int)b, (unsigned int)node,
-                                       (unsigned int)stream_id, (unsigned int)seed, (unsigned int)(seed >> 32));
+                                       (unsigned int)stream_id + 2u * (unsigned int)(offset >> 32),
+                                       (unsigned int)seed, (unsigned int)(seed >> 32));
     return (float)(x0 >> 8) * 5.9604644775390625e-8f;  // 2^-24
 }
 
@@ -153,5 +166,6 @@ hs_status hs_launch_accept(hs_ctx* ctx, const hs_tree_batch* tree, const hs_prun
                            hs_dtype dtype, int64_t row_stride, int32_t vocab, const int32_t* mode,
                            const float* temperature, uint64_t seed, uint64_t offset, const float* uniforms,
                            const hs_accept_out* out, cudaStream_t stream);
+hs_status hs_launch_wait_selftest(hs_ctx* ctx, uint64_t limit_ns, cudaStream_t stream);
 hs_status hs_launch_philox(uint64_t seed, uint64_t offset, const int32_t* b, const int32_t* node,
                            const int32_t* stream_id, int32_t count, float* out, cudaStream_t stream);

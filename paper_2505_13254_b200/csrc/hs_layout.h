@@ -33,4 +33,3 @@ static inline int hs_row_chunks(int32_t vocab, hs_dtype dt) {
 // per (row, chunk) partial of the accept pass: {argmax key (8 bytes), max, sum e}
 #define HS_ACC_PARTIAL_BYTES 16
 
-#define HS_ATTN_WS_SPLITS 8

@@ -41,18 +41,22 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned int bar, unsigned int par
 }
 // Bounded wait: polls until the phase with the given parity has completed or HS_WAIT_LIMIT_NS have
 // passed; on expiry records HS_ERR_TIMEOUT in *err and returns false.  Never spins forever.
-__device__ __forceinline__ bool mbar_wait(unsigned int bar, unsigned int parity, int* err) {
+__device__ __forceinline__ bool mbar_wait_limit(unsigned int bar, unsigned int parity, int* err,
+                                                unsigned long long limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
     for (;;) {
 #pragma unroll 1
         for (int i = 0; i < 128; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (global_timer_ns() - t0 > HS_WAIT_LIMIT_NS) {
+        if (global_timer_ns() - t0 > limit_ns) {
             atomicExch(err, (int)HS_ERR_TIMEOUT);
             return false;
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(unsigned int bar, unsigned int parity, int* err) {
+    return mbar_wait_limit(bar, parity, err, HS_WAIT_LIMIT_NS);
 }
 
 // Untiled bulk copy global -> shared (both 16-byte aligned, size a multiple of 16), completion

@@ -1,18 +1,21 @@
-// hs_entropy_quantify: one launch.
+// hs_entropy_quantify: two launches.
 //
-// Stage 1 (every CTA): a CTA owns one chunk of one logits row (up to 32 KiB), brings it on chip in
-// one piece and reduces max / sum e^x / sum x e^x with warp shuffles.  Staged variant (the default):
-// one bulk copy into shared memory, issued by one thread before the dependency wait; the passes read
-// shared memory, so a thread needs few registers and four CTAs share an SM (at one tree every CTA of
-// the launch is resident at once: no row waits for a second wave).  Register variant (the
-// allocation-free entry point, and rows a caller of the launcher hands over unaligned: the C entry
-// point rejects those): 16-byte coalesced loads that are all issued before the first use, two CTAs per SM.  The Top-K of the chunk is found without sorting: the K-th largest of 32 group maxima
-// is a lower bound of the chunk's K-th largest logit, only threads whose own maximum reaches it
-// re-scan their registers, and the few candidates are ranked by counting.
-// Stage 2 (last CTA of a row to arrive): merges the row's chunk partials into max, log-sum-exp,
-// Shannon entropy, Top-K and the two Top-K entropies (Eq. 1 inner sum).
-// Stage 3 (last row of a tree to arrive): path confidence ln V_i (Sec. 2.2), cumulative
-// meta-path Top-K entropy Phi (Eq. 1) and the operational path P* (Sec. 4.1) of that tree.
+// quantify_stream_kernel   The logits matrix is one long stream of 16-byte vectors (row after row) that is cut
+//     into equal contiguous shares, one per CTA, one CTA per SM.  A producer warp brings the share on chip in
+//     items of up to 32 KiB (bulk copies into a ring of shared-memory slots, completion on mbarriers); sixteen
+//     consumer warps reduce each item in ONE pass: running maximum per thread (packed bf16 maxima), then
+//     sum e^(x-m) and sum x e^(x-m) with the exponent's multiply-add and the two sums as packed fp32 pairs.
+//     Top-K without sorting: after every window of three items a warp takes a lower bound of the K-th
+//     largest logit of the row share from maxima of disjoint element sets (the 32 half-warp maxima of the
+//     CTA, or its own 32 lane maxima on a short share), and only lanes whose window maximum reaches the bound
+//     re-scan their vectors in shared memory and push candidates; the few candidates are ranked by counting.
+//     A share that ends inside a row leaves a partial {max, sum, sum x e, K keys}; the last CTA of a row to
+//     arrive merges the partials into max, log-sum-exp, Shannon entropy, Top-K and the two Top-K entropies
+//     (Eq. 1 inner sum).  Rows that lie inside one share need no partial and no atomic.
+// tree_scores_kernel       One CTA per sequence: path confidence ln V_i (Sec. 2.2), cumulative meta-path
+//     Top-K entropy Phi (Eq. 1) and the operational path P* (Sec. 4.1).
+//
+// quantify_chunk_kernel (a CTA owns one chunk of one row, registers only) serves the allocation-free entry.
 #include <math_constants.h>
 
 #include <mutex>
@@ -24,24 +27,34 @@
 #define CAND_CAP 512
 #define LOG2E 1.4426950408889634f
 
+#define QS_CONSUMERS 512                      // sixteen consumer warps
+#define QS_THREADS (QS_CONSUMERS + 32)        // + the producer warp
+#define QS_ITEM_VECS 2048                     // vectors per item: 32 KiB, four per consumer thread
+#define QS_VPT (QS_ITEM_VECS / QS_CONSUMERS)
+#define QS_SLOTS 6                            // ring of item slots
+#define QS_WINDOW 3                           // items a consumer holds before it hands their slots back
+#define QS_MAX_SEGS 32                        // shares a row may be split over
+#define QS_SMEM_BYTES (QS_SLOTS * QS_ITEM_VECS * 16 + 128)
+
 struct QuantParams {
     const void* logits;
     int64_t row_stride;
     int vocab;
     int nvec;        // 16-byte vectors per row, the last one may be partial
-    int chunks;      // CTAs per row
-    int chunk_vecs;  // vectors per chunk
+    int chunks;      // chunk kernel: CTAs per row
+    int chunk_vecs;  // chunk kernel: vectors per chunk
+    int per;         // stream kernel: vectors per CTA share
     int rows;
     int batch;
     const int* node_off;
     const int* parent;
     const int* token;
     hs_quant_out out;
-    float4* part_stats;             // [rows*chunks] {max, sum e, sum e*x, -}
-    unsigned long long* part_keys;  // [rows*chunks*HS_MAX_TOPK]
+    float4* part_stats;             // {max, sum e, sum e*x, -} per partial
+    unsigned long long* part_keys;  // HS_MAX_TOPK keys per partial
     int* row_cnt;
-    int* tree_cnt;
     int K, d_base, phi_mode, pstar_mode, entropy_mode, is_bf16;
+    int prefetch;    // the rows may be fetched before the dependency wait (the caller vouches that they are complete)
     int* err;        // sticky device error word (a bounded wait that expired)
 };
 
@@ -62,10 +75,10 @@ __device__ __forceinline__ float ex2f(float x) {
     return y;
 }
 
-// Rank candidates s_cand[0..n) by key (all distinct, 0 = empty) and write the K best to s_top.
+// Rank candidates s_cand[0..n) by key (all distinct, 0 = empty) and write the K best to s_top (zeroed before).
 __device__ __forceinline__ void rank_select(const unsigned long long* s_cand, int n, int K,
-                                            unsigned long long* s_top) {
-    for (int t = threadIdx.x; t < n; t += blockDim.x) {
+                                            unsigned long long* s_top, int tid, int nthr) {
+    for (int t = tid; t < n; t += nthr) {
         unsigned long long k = s_cand[t];
         if (k == 0ull) continue;
         int rank = 0;
@@ -74,23 +87,30 @@ __device__ __forceinline__ void rank_select(const unsigned long long* s_cand, in
     }
 }
 
-// Cold path of the chunk Top-K: K block-wide arg-max rounds over the chunk, each restricted to keys
-// below the previous winner.  Exact for any number of ties.
+// barrier over the first `nthr` threads of the CTA (a multiple of 32); id 0 is __syncthreads' own
+__device__ __forceinline__ void bar_sync(int id, int nthr) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthr) : "memory");
+}
+
+// Cold path of the Top-K: K rounds of "largest key below the previous winner" over vectors [v0, v1) of a row,
+// read from global memory by `nthr` threads (barrier `bar`).  Exact for any number of ties; -inf logits are no
+// candidates.  s_red: one slot per warp.
 template <bool BF16>
 __device__ __noinline__ void topk_by_rounds(const char* rowp, int v0, int v1, int vocab, int K,
-                                            unsigned long long* s_top, unsigned long long* s_red) {
+                                            unsigned long long* s_top, unsigned long long* s_red,
+                                            int tid, int nthr, int bar) {
     constexpr int VE = BF16 ? 8 : 4;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
     unsigned long long last = ~0ull;
     for (int r = 0; r < K; ++r) {
         unsigned long long best = 0ull;
-        for (int v = v0 + tid; v < v1; v += HS_ROW_THREADS) {
+        for (int v = v0 + tid; v < v1; v += nthr) {
             uint4 dv = __ldg((const uint4*)(rowp) + v);
             float x[8];
             unpack<BF16>(dv, x);
 #pragma unroll
             for (int e = 0; e < VE; ++e) {
-                if (v * VE + e < vocab) {
+                if (v * VE + e < vocab && x[e] > -CUDART_INF_F) {
                     unsigned long long k = make_key(x[e], v * VE + e);
                     if (k < last && k > best) best = k;
                 }
@@ -98,26 +118,530 @@ __device__ __noinline__ void topk_by_rounds(const char* rowp, int v0, int v1, in
         }
         best = warp_max_u64(best);
         if (lane == 0) s_red[warp] = best;
-        __syncthreads();
+        bar_sync(bar, nthr);
         best = s_red[0];
-        for (int w = 1; w < 8; ++w) best = s_red[w] > best ? s_red[w] : best;
+        for (int w = 1; w < nwarp; ++w) best = s_red[w] > best ? s_red[w] : best;
         if (tid == 0) s_top[r] = best;
         last = best;
-        __syncthreads();
+        bar_sync(bar, nthr);
         if (best == 0ull) break;
     }
 }
 
-__device__ void tree_scores(const QuantParams& p, int b, float* s_f, int* s_i);
+// One warp: the statistics of a whole row from its {max, sum e^(x-max), sum x e^(x-max)} and its K best keys
+// (s_top, 0 = none): log-sum-exp, Shannon entropy, Top-K values and token ids, the entropy of the renormalised
+// Top-K probabilities (Eq. 1 inner sum) and the truncated variant.
+__device__ __forceinline__ void finalize_row(const QuantParams& p, int row, float M, float S, float U,
+                                             const unsigned long long* s_top, int lane) {
+    const int K = p.K;
+    const float lse = M + logf(S);
+    const float H = lse - U / S;
+    const unsigned long long key = (lane < K) ? s_top[lane] : 0ull;
+    const bool valid = key != 0ull;
+    const float tv = valid ? key_value(key) : 0.f;
+    const float t0 = __shfl_sync(HS_FULL_MASK, tv, 0);
+    const float pv = valid ? expf(tv - lse) : 0.f;
+    const float itr = warp_sum(valid ? -pv * (tv - lse) : 0.f);
+    const float z = valid ? expf(tv - t0) : 0.f;
+    const float Z = warp_sum(z);
+    const float itk = logf(Z) - warp_sum(valid ? z * (tv - t0) : 0.f) / Z;
+    if (lane < K) {
+        p.out.topk_val[(size_t)row * K + lane] = valid ? tv : -CUDART_INF_F;
+        p.out.topk_idx[(size_t)row * K + lane] = valid ? key_index(key) : -1;
+    }
+    if (lane == 0) {
+        p.out.row_max[row] = M;
+        p.out.row_lse[row] = lse;
+        p.out.h_full[row] = fmaxf(H, 0.f);
+        p.out.i_topk[row] = fmaxf(itk, 0.f);
+        p.out.i_trunc[row] = itr;
+    }
+}
 
-// MODE 0: register variant; 1: staged, loops over the vectors unrolled; 2: staged, loops rolled
-template <bool BF16, int MODE>
-__global__ void __launch_bounds__(HS_ROW_THREADS, MODE ? 4 : 2) quantify_kernel(const QuantParams p) {
-    constexpr bool STAGED = MODE != 0;
+// K-th largest of the warp's 32 values (one per lane), -inf if fewer than K are above -inf.  K rounds of a
+// warp-wide maximum that retires one holder of the maximum per round (ties count one by one).
+__device__ __forceinline__ float warp_kth_largest(float v, int K, int lane) {
+    unsigned int ob = (v > -CUDART_INF_F) ? float_order_bits(v) : 0u;
+    unsigned int mx = 0u;
+    for (int i = 0; i < K; ++i) {
+        mx = __reduce_max_sync(HS_FULL_MASK, ob);
+        const unsigned int holders = __ballot_sync(HS_FULL_MASK, ob == mx);
+        if (lane == __ffs(holders) - 1) ob = 0u;
+    }
+    return mx ? order_bits_float(mx) : -CUDART_INF_F;
+}
+
+// ================================================================================================================
+// The streaming kernel
+// ================================================================================================================
+template <bool BF16>
+__global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const QuantParams p) {
+    constexpr int VE = BF16 ? 8 : 4;
+    extern __shared__ __align__(128) unsigned char s_dyn[];
+    __shared__ unsigned long long s_full[QS_SLOTS], s_empty[QS_SLOTS];
+    __shared__ unsigned long long s_list[CAND_CAP];
+    __shared__ unsigned long long s_top[HS_MAX_TOPK];
+    __shared__ unsigned long long s_red[QS_CONSUMERS / 32];
+    __shared__ float s_gm[32];
+    __shared__ float s_wstat[QS_CONSUMERS / 32][3];
+    __shared__ int s_cnt;
+    __shared__ int s_flag;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const unsigned int slots0 = (smem_u32(s_dyn) + 127u) & ~127u;
+    const unsigned char* slots_gen = s_dyn + (slots0 - smem_u32(s_dyn));
+    const long long total = (long long)p.rows * p.nvec;
+    const long long g0 = (long long)blockIdx.x * p.per;
+    const long long g1 = min(g0 + (long long)p.per, total);
+    const size_t esz = BF16 ? 2 : 4;
+
+    if (tid == 0) {
+        for (int s = 0; s < QS_SLOTS; ++s) {
+            mbar_init(smem_u32(&s_full[s]), 1);
+            mbar_init(smem_u32(&s_empty[s]), QS_CONSUMERS / 32);
+        }
+        mbar_init_fence();
+        s_cnt = 0;
+    }
+    if (tid < HS_MAX_TOPK) s_top[tid] = 0ull;
+    __syncthreads();
+    pdl_launch_dependents();
+
+    if (warp == QS_CONSUMERS / 32) {
+        // ---- producer: one lane walks the share item by item ----------------------------------------------------
+        if (lane == 0) {
+            long long g = g0;
+            int it = 0;
+            bool waited = false;
+            if (!p.prefetch) { pdl_wait(); waited = true; }
+            while (g < g1) {
+                const int row = (int)(g / p.nvec);
+                const int v = (int)(g - (long long)row * p.nvec);
+                const int len = (int)min((long long)min(QS_ITEM_VECS, p.nvec - v), g1 - g);
+                const int slot = it % QS_SLOTS;
+                if (it >= QS_SLOTS) {
+                    if (!waited) { pdl_wait(); waited = true; }     // (nothing of this kernel is written by the producer)
+                    mbar_wait(smem_u32(&s_empty[slot]), (unsigned int)(it / QS_SLOTS - 1) & 1u, p.err);
+                }
+                const unsigned int bar = smem_u32(&s_full[slot]);
+                mbar_expect_tx(bar, (unsigned int)len * 16u);
+                bulk_load(slots0 + (unsigned int)slot * (QS_ITEM_VECS * 16),
+                          (const char*)p.logits + (size_t)row * p.row_stride * esz + (size_t)v * 16, (unsigned int)len * 16u, bar);
+                g += len;
+                ++it;
+            }
+        }
+        return;
+    }
+
+    // ---- consumers -------------------------------------------------------------------------------------------------
+    pdl_wait();                    // partials, counters and outputs may still be in use by the kernel ahead
+    const int K = p.K;
+    const unsigned int ninf = BF16 ? 0xff80ff80u : 0xff800000u;
+    const unsigned int floor2 = 0xf149f149u;     // bf16 pair of -1e30: keeps 0 * x finite for x = -inf
+    int it = 0;
+    long long g = g0;
+    while (g < g1) {
+        // ---- one segment: the part [g, seg_end) of this share inside row `row` ------------------------------------
+        const int row = (int)(g / p.nvec);
+        const long long row_g0 = (long long)row * p.nvec;
+        const int sv0 = (int)(g - row_g0);
+        const int sv1 = (int)(min(g1, row_g0 + p.nvec) - row_g0);
+        const char* rowp = (const char*)p.logits + (size_t)row * p.row_stride * esz;
+        float m_t = -CUDART_INF_F;                // running maximum of this thread's logits of the segment
+        float2 s2 = make_float2(0.f, 0.f), u2 = make_float2(0.f, 0.f);
+        float tau = -CUDART_INF_F;                // lower bound of the K-th largest logit of the segment
+        int v = sv0;
+        bool first_window = true;
+        while (v < sv1) {
+            // ---- a window of up to QS_WINDOW items -------------------------------------------------------------
+            float vmx[QS_WINDOW * QS_VPT];
+            int w_slot[QS_WINDOW], w_v0[QS_WINDOW], w_len[QS_WINDOW];
+            int nitems = 0;
+            float wmax = -CUDART_INF_F;
+            const int win_v0 = v;
+#pragma unroll
+            for (int wi = 0; wi < QS_WINDOW; ++wi) {
+#pragma unroll
+                for (int j = 0; j < QS_VPT; ++j) vmx[wi * QS_VPT + j] = -CUDART_INF_F;
+                w_slot[wi] = 0; w_v0[wi] = 0; w_len[wi] = 0;
+                if (v < sv1) {
+                    const int len = min(QS_ITEM_VECS, sv1 - v);
+                    const int slot = it % QS_SLOTS;
+                    w_slot[wi] = slot; w_v0[wi] = v; w_len[wi] = len;
+                    nitems = wi + 1;
+                    mbar_wait(smem_u32(&s_full[slot]), (unsigned int)(it / QS_SLOTS) & 1u, p.err);
+                    const uint4* st = reinterpret_cast<const uint4*>(slots_gen + (size_t)slot * (QS_ITEM_VECS * 16));
+                    uint4 d[QS_VPT];
+                    float imax = -CUDART_INF_F;
+#pragma unroll
+                    for (int j = 0; j < QS_VPT; ++j) {
+                        const int vl = tid + j * QS_CONSUMERS;
+                        d[j] = (vl < len) ? st[vl] : make_uint4(ninf, ninf, ninf, ninf);
+                        if (v + vl == p.nvec - 1 && p.nvec * VE != p.vocab) {      // the row's last vector runs past vocab
+                            unsigned int* wd = reinterpret_cast<unsigned int*>(&d[j]);
+#pragma unroll
+                            for (int e = 0; e < VE; ++e)
+                                if ((p.nvec - 1) * VE + e >= p.vocab) {
+                                    if (BF16) wd[e >> 1] = (e & 1) ? ((wd[e >> 1] & 0x0000ffffu) | 0xff800000u)
+                                                                   : ((wd[e >> 1] & 0xffff0000u) | 0x0000ff80u);
+                                    else wd[e] = 0xff800000u;
+                                }
+                        }
+                        float vm;
+                        if (BF16) {
+                            const __nv_bfloat162 a = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&d[j].x),
+                                                            *reinterpret_cast<const __nv_bfloat162*>(&d[j].y));
+                            const __nv_bfloat162 b = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&d[j].z),
+                                                            *reinterpret_cast<const __nv_bfloat162*>(&d[j].w));
+                            const __nv_bfloat162 c = __hmax2(a, b);
+                            const unsigned int cw = *reinterpret_cast<const unsigned int*>(&c);
+                            vm = fmaxf(bf16_lo(cw), bf16_hi(cw));
+                        } else {
+                            vm = fmaxf(fmaxf(__uint_as_float(d[j].x), __uint_as_float(d[j].y)),
+                                       fmaxf(__uint_as_float(d[j].z), __uint_as_float(d[j].w)));
+                        }
+                        vmx[wi * QS_VPT + j] = vm;
+                        imax = fmaxf(imax, vm);
+                    }
+                    if (imax > m_t) {                         // the thread's maximum grows: rescale its sums
+                        const float f = (m_t == -CUDART_INF_F) ? 0.f : ex2f((m_t - imax) * LOG2E);
+                        s2.x *= f; s2.y *= f; u2.x *= f; u2.y *= f;
+                        m_t = imax;
+                    }
+                    wmax = fmaxf(wmax, imax);
+                    const float nml = (m_t == -CUDART_INF_F) ? 0.f : -m_t * LOG2E;
+                    const float2 l2 = make_float2(LOG2E, LOG2E), n2 = make_float2(nml, nml);
+#pragma unroll
+                    for (int j = 0; j < QS_VPT; ++j) {
+                        if (BF16) {
+                            const unsigned int* wd = reinterpret_cast<const unsigned int*>(&d[j]);
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const __nv_bfloat162 cl = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&wd[q]),
+                                                                 *reinterpret_cast<const __nv_bfloat162*>(&floor2));
+                                const unsigned int cw = *reinterpret_cast<const unsigned int*>(&cl);
+                                const float2 x = make_float2(bf16_lo(cw), bf16_hi(cw));
+                                const float2 t = fma2_ftz(x, l2, n2);
+                                const float2 e = make_float2(ex2f(t.x), ex2f(t.y));
+                                s2 = add2_ftz(s2, e);
+                                u2 = fma2_ftz(e, x, u2);
+                            }
+                        } else {
+                            const unsigned int* wd = reinterpret_cast<const unsigned int*>(&d[j]);
+#pragma unroll
+                            for (int q = 0; q < 2; ++q) {
+                                const float2 x = make_float2(fmaxf(__uint_as_float(wd[2 * q]), -1e30f),
+                                                             fmaxf(__uint_as_float(wd[2 * q + 1]), -1e30f));
+                                const float2 t = fma2_ftz(x, l2, n2);
+                                const float2 e = make_float2(ex2f(t.x), ex2f(t.y));
+                                s2 = add2_ftz(s2, e);
+                                u2 = fma2_ftz(e, x, u2);
+                            }
+                        }
+                    }
+                    v += len;
+                    ++it;
+                }
+            }
+            // ---- a lower bound of the segment's K-th largest logit -------------------------------------------
+            // Maxima of disjoint element sets are distinct elements, so the K-th largest of any such family is a
+            // bound.  A window of at least one full item: the CTA's 32 half-warp maxima (published in shared memory;
+            // an entry another warp has not refreshed yet is an older maximum of the same segment, still an element
+            // of it).  Shorter: this warp's own 32 lane maxima.
+            const int win_vecs = v - win_v0;
+            if (win_vecs >= QS_ITEM_VECS) {
+                float hm = m_t;
+                hm = fmaxf(hm, __shfl_xor_sync(HS_FULL_MASK, hm, 1));
+                hm = fmaxf(hm, __shfl_xor_sync(HS_FULL_MASK, hm, 2));
+                hm = fmaxf(hm, __shfl_xor_sync(HS_FULL_MASK, hm, 4));
+                hm = fmaxf(hm, __shfl_xor_sync(HS_FULL_MASK, hm, 8));
+                if ((lane & 15) == 0) s_gm[warp * 2 + (lane >> 4)] = hm;
+                if (first_window) bar_sync(1, QS_CONSUMERS);      // every warp has published maxima of this segment
+                else __syncwarp();
+                tau = fmaxf(tau, warp_kth_largest(s_gm[lane], K, lane));
+            } else {
+                if (first_window) bar_sync(1, QS_CONSUMERS);      // (keeps the barrier count the same for every warp)
+                tau = fmaxf(tau, warp_kth_largest(m_t, K, lane));
+            }
+            first_window = false;
+            // ---- candidates: lanes whose window maximum reaches the bound re-scan their vectors ------------------
+            if (wmax >= tau && wmax > -CUDART_INF_F) {
+#pragma unroll 1
+                for (int i = 0; i < nitems * QS_VPT; ++i) {
+                    float vm = -CUDART_INF_F;
+#pragma unroll
+                    for (int q = 0; q < QS_WINDOW * QS_VPT; ++q) vm = (q == i) ? vmx[q] : vm;
+                    if (vm >= tau && vm > -CUDART_INF_F) {
+                        const int wi = i / QS_VPT, j = i - wi * QS_VPT;
+                        int slot = 0, iv0 = 0;
+#pragma unroll
+                        for (int q = 0; q < QS_WINDOW; ++q) { slot = (q == wi) ? w_slot[q] : slot; iv0 = (q == wi) ? w_v0[q] : iv0; }
+                        const int vl = tid + j * QS_CONSUMERS;
+                        const uint4 dv = reinterpret_cast<const uint4*>(slots_gen + (size_t)slot * (QS_ITEM_VECS * 16))[vl];
+                        float x[8];
+                        unpack<BF16>(dv, x);
+                        const int base = (iv0 + vl) * VE;
+#pragma unroll
+                        for (int e = 0; e < VE; ++e) {
+                            if (x[e] >= tau && x[e] > -CUDART_INF_F && base + e < p.vocab) {
+                                const int sl = atomicAdd(&s_cnt, 1);
+                                if (sl < CAND_CAP) s_list[sl] = make_key(x[e], base + e);
+                            }
+                        }
+                    }
+                }
+            }
+            // ---- the window's slots go back to the producer -------------------------------------------------------
+            __syncwarp();
+            if (lane == 0)
+                for (int wi = 0; wi < nitems; ++wi) {
+                    int slot = 0;
+#pragma unroll
+                    for (int q = 0; q < QS_WINDOW; ++q) slot = (q == wi) ? w_slot[q] : slot;
+                    mbar_arrive(smem_u32(&s_empty[slot]));
+                }
+        }
+        // ---- end of the segment: warp, then CTA reduction of (max, s, u); Top-K of the candidates ------------------
+        {
+            const float wm = warp_max(m_t);
+            const float f = (m_t == -CUDART_INF_F) ? 0.f : ex2f((m_t - wm) * LOG2E);
+            const float ws = warp_sum((s2.x + s2.y) * f), wu = warp_sum((u2.x + u2.y) * f);
+            if (lane == 0) { s_wstat[warp][0] = wm; s_wstat[warp][1] = ws; s_wstat[warp][2] = wu; }
+        }
+        bar_sync(1, QS_CONSUMERS);                    // all candidates are pushed, all warp sums written
+        const int ncand = s_cnt;
+        if (ncand <= CAND_CAP) rank_select(s_list, ncand, K, s_top, tid, QS_CONSUMERS);
+        else topk_by_rounds<BF16>(rowp, sv0, sv1, p.vocab, K, s_top, s_red, tid, QS_CONSUMERS, 1);   // heavy ties
+        bar_sync(1, QS_CONSUMERS);                    // s_top is complete
+        // segments of this row: shares c_first .. c_last
+        const int c_first = (int)(row_g0 / p.per), c_last = (int)((row_g0 + p.nvec - 1) / p.per);
+        const int nseg = c_last - c_first + 1;
+        if (warp == 0) {
+            // the sixteen warps' (max, s, u) in a fixed order
+            const float wm = lane < QS_CONSUMERS / 32 ? s_wstat[lane & 15][0] : -CUDART_INF_F;
+            const float M = warp_max(wm);
+            const float f = (lane >= QS_CONSUMERS / 32 || wm == -CUDART_INF_F) ? 0.f : ex2f((wm - M) * LOG2E);
+            const float S = s_wstat[lane & 15][1] * f, U = s_wstat[lane & 15][2] * f;
+            float St = 0.f, Ut = 0.f;
+#pragma unroll
+            for (int w = 0; w < QS_CONSUMERS / 32; ++w) {
+                St += __shfl_sync(HS_FULL_MASK, S, w);
+                Ut += __shfl_sync(HS_FULL_MASK, U, w);
+            }
+            if (nseg == 1) {
+                finalize_row(p, row, M, St, Ut, s_top, lane);
+                if (lane == 0) { s_flag = 0; s_cnt = 0; }
+            } else {
+                // partial slot: two per share, the leading one for a row that began in an earlier share
+                const int ps = 2 * blockIdx.x + (row_g0 < g0 ? 0 : 1);
+                if (lane == 0) p.part_stats[ps] = make_float4(M, St, Ut, 0.f);
+                if (lane < HS_MAX_TOPK) p.part_keys[(size_t)ps * HS_MAX_TOPK + lane] = (lane < K) ? s_top[lane] : 0ull;
+                __syncwarp();
+                if (lane == 0) {
+                    __threadfence();
+                    const int last = atomicAdd(&p.row_cnt[row], 1) == nseg - 1;
+                    if (last) p.row_cnt[row] = 0;              // ready for the next launch
+                    __threadfence();
+                    s_flag = last;
+                    s_cnt = 0;
+                }
+            }
+        }
+        bar_sync(1, QS_CONSUMERS);                    // s_flag; s_top and s_list may be reused
+        if (s_flag) {
+            // ---- the last share of a split row merges the row's partials -------------------------------------------
+            if (tid < HS_MAX_TOPK) s_top[tid] = 0ull;
+            for (int t = tid; t < nseg * HS_MAX_TOPK; t += QS_CONSUMERS) {
+                const int c = c_first + t / HS_MAX_TOPK;
+                const int ps = 2 * c + (row_g0 < (long long)c * p.per ? 0 : 1);
+                s_list[t] = __ldcg(&p.part_keys[(size_t)ps * HS_MAX_TOPK + (t % HS_MAX_TOPK)]);
+            }
+            bar_sync(1, QS_CONSUMERS);
+            rank_select(s_list, nseg * HS_MAX_TOPK, K, s_top, tid, QS_CONSUMERS);
+            bar_sync(1, QS_CONSUMERS);
+            if (warp == 0) {
+                float m = -CUDART_INF_F, cs = 0.f, cu = 0.f;
+                if (lane < nseg) {
+                    const int c = c_first + lane;
+                    const int ps = 2 * c + (row_g0 < (long long)c * p.per ? 0 : 1);
+                    const float4 stv = __ldcg(&p.part_stats[ps]);
+                    m = stv.x; cs = stv.y; cu = stv.z;
+                }
+                const float M = warp_max(m);
+                const float f = (m == -CUDART_INF_F) ? 0.f : ex2f((m - M) * LOG2E);
+                const float S = warp_sum(cs * f), U = warp_sum(cu * f);
+                finalize_row(p, row, M, S, U, s_top, lane);
+            }
+            bar_sync(1, QS_CONSUMERS);
+        }
+        if (tid < HS_MAX_TOPK) s_top[tid] = 0ull;     // (next written after the next segment's first barrier)
+        g = row_g0 + sv1;
+    }
+}
+
+// ================================================================================================================
+// Tree stage: one CTA of 128 threads per sequence, one thread per node
+// ================================================================================================================
+__global__ void __launch_bounds__(HS_MAX_NODES) tree_scores_kernel(const QuantParams p) {
+    __shared__ float s_logc[HS_MAX_NODES], s_I[HS_MAX_NODES], s_phi[HS_MAX_NODES];
+    __shared__ int s_par[HS_MAX_NODES];
+    __shared__ unsigned long long s_best[4];
+    __shared__ int s_maxd[4];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = blockIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();                                   // the row statistics come from the kernel ahead
+    const int base = p.node_off[b];
+    const int n = p.node_off[b + 1] - base;
+    // validation
+    int bad = (n > HS_MAX_NODES || n <= 0);
+    int par = -1, tok = 0;
+    if (!bad && tid < n) {
+        par = p.parent[base + tid];
+        tok = p.token[base + tid];
+        if (tid == 0) bad = (par != -1);
+        else bad = (par < 0 || par >= tid || tok < 0 || tok >= p.vocab);
+    }
+    bad = __syncthreads_or(bad);
+    if (bad) {
+        for (int i = tid; i < n; i += blockDim.x) {
+            p.out.logc[base + i] = 0.f; p.out.score[base + i] = 0.f; p.out.phi[base + i] = 0.f;
+            p.out.depth[base + i] = 0;
+        }
+        if (tid == 0) { p.out.status[b] = HS_ERR_BAD_TREE; p.out.pstar_node[b] = 0; p.out.phi_star[b] = 0.f; }
+        return;
+    }
+    if (tid < n) {
+        float lc = 0.f;
+        if (tid > 0) {
+            const size_t off = (size_t)(base + par) * p.row_stride + tok;
+            const float lv = p.is_bf16 ? __bfloat162float(((const __nv_bfloat16*)p.logits)[off])
+                                       : ((const float*)p.logits)[off];
+            lc = lv - p.out.row_lse[base + par];
+        }
+        s_logc[tid] = lc;
+        s_I[tid] = p.entropy_mode == 0 ? p.out.i_topk[base + tid] : p.out.i_trunc[base + tid];
+        s_par[tid] = par;
+    }
+    __syncthreads();
+    float S = 0.f, Phi = 0.f;
+    int dep = 0;
+    if (tid < n) {
+        int a = tid;
+        while (a > 0) {
+            const int pa = s_par[a];
+            S += s_logc[a];
+            Phi += s_I[pa];
+            a = pa;
+            ++dep;
+        }
+        if (p.phi_mode == 1) Phi += s_I[tid];
+        s_phi[tid] = Phi;
+        p.out.logc[base + tid] = s_logc[tid];
+        p.out.score[base + tid] = S;
+        p.out.phi[base + tid] = Phi;
+        p.out.depth[base + tid] = dep;
+    }
+    // deepest level, then P* among the nodes of depth min(d_base, deepest)
+    int md = dep;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) md = max(md, __shfl_xor_sync(HS_FULL_MASK, md, o));
+    if (lane == 0) s_maxd[warp] = md;
+    __syncthreads();
+    md = max(max(s_maxd[0], s_maxd[1]), max(s_maxd[2], s_maxd[3]));
+    const int t_eval = min(p.d_base, md);
+    unsigned long long key = 0ull;
+    if (tid < n && dep == t_eval) key = make_key(p.pstar_mode == 0 ? s_logc[tid] : S, tid);
+    key = warp_max_u64(key);
+    if (lane == 0) s_best[warp] = key;
+    __syncthreads();
+    if (tid == 0) {
+        unsigned long long best = s_best[0];
+        for (int w = 1; w < 4; ++w) best = s_best[w] > best ? s_best[w] : best;
+        const int node = key_index(best);
+        p.out.pstar_node[b] = node;
+        p.out.phi_star[b] = s_phi[node];
+        p.out.status[b] = HS_OK;
+    }
+}
+
+static void fill_common(QuantParams& p, const hs_tree_batch* tree, const void* logits, hs_dtype dtype,
+                        int64_t row_stride, int32_t vocab, const hs_policy* policy, const hs_quant_out* out) {
+    const int ve = hs_vec_elems(dtype);
+    p.logits = logits;
+    p.row_stride = row_stride;
+    p.vocab = vocab;
+    p.nvec = (vocab + ve - 1) / ve;
+    p.chunks = 0;
+    p.chunk_vecs = 0;
+    p.per = 0;
+    p.rows = tree->n_nodes_total;
+    p.batch = tree->batch;
+    p.node_off = tree->node_off;
+    p.parent = tree->parent;
+    p.token = tree->token;
+    p.out = *out;
+    p.K = policy->top_k;
+    p.d_base = policy->d_base;
+    p.phi_mode = policy->phi_mode;
+    p.pstar_mode = policy->pstar_mode;
+    p.entropy_mode = policy->entropy_mode;
+    p.is_bf16 = dtype == HS_BF16;
+    p.prefetch = 0;
+    p.err = nullptr;
+}
+
+// Shares of the stream: at most one per SM, at least 32 KiB each, and so large that no row is split over more
+// than QS_MAX_SEGS of them.
+static int quantify_share_vecs(long long total_vecs, int nvec, int sm_count) {
+    long long per = (total_vecs + sm_count - 1) / sm_count;
+    const long long floor_row = (nvec + (QS_MAX_SEGS - 2) - 1) / (QS_MAX_SEGS - 2);
+    if (per < floor_row) per = floor_row;
+    if (per < QS_ITEM_VECS) per = QS_ITEM_VECS;
+    return (int)per;
+}
+
+hs_status hs_launch_quantify(hs_ctx* ctx, const hs_tree_batch* tree, const void* logits, hs_dtype dtype,
+                             int64_t row_stride, int32_t vocab, const hs_policy* policy,
+                             const hs_quant_out* out, cudaStream_t stream) {
+    QuantParams p;
+    fill_common(p, tree, logits, dtype, row_stride, vocab, policy, out);
+    if (p.nvec > QS_ITEM_VECS * 64) return HS_ERR_SHAPE;            // vocabulary beyond 2^20 bf16 / 2^19 fp32 logits
+    const long long total = (long long)p.rows * p.nvec;
+    p.per = quantify_share_vecs(total, p.nvec, ctx->sm_count);
+    const int nctas = (int)((total + p.per - 1) / p.per);
+    const size_t stats_bytes = hs_align_up((size_t)2 * nctas * sizeof(float4), 256);
+    const size_t keys_bytes = (size_t)2 * nctas * HS_MAX_TOPK * sizeof(unsigned long long);
+    if (stats_bytes + keys_bytes > ctx->scratch_bytes) return HS_ERR_WORKSPACE;
+    p.part_stats = (float4*)ctx->scratch;
+    p.part_keys = (unsigned long long*)(ctx->scratch + stats_bytes);
+    p.row_cnt = ctx->counters + HS_CNT_QUANT_ROW;
+    p.err = ctx->counters + HS_CNT_ERROR;
+    p.prefetch = (ctx->prefetch & HS_PREFETCH_LOGITS) != 0;
+    if (!ctx->quant_ready) {
+        if (cudaFuncSetAttribute(quantify_stream_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, QS_SMEM_BYTES) != cudaSuccess ||
+            cudaFuncSetAttribute(quantify_stream_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, QS_SMEM_BYTES) != cudaSuccess)
+            return HS_ERR_CUDA;
+        ctx->quant_ready = true;
+    }
+    cudaError_t e = dtype == HS_BF16
+        ? hs_launch(quantify_stream_kernel<true>, dim3(nctas), dim3(QS_THREADS), QS_SMEM_BYTES, stream, ctx->pdl, dim3(1, 1, 1), p)
+        : hs_launch(quantify_stream_kernel<false>, dim3(nctas), dim3(QS_THREADS), QS_SMEM_BYTES, stream, ctx->pdl, dim3(1, 1, 1), p);
+    if (e != cudaSuccess) return HS_ERR_CUDA;
+    e = hs_launch(tree_scores_kernel, dim3(p.batch), dim3(HS_MAX_NODES), 0, stream, ctx->pdl, dim3(1, 1, 1), p);
+    return e == cudaSuccess ? HS_OK : HS_ERR_CUDA;
+}
+
+// ================================================================================================================
+// The chunk kernel: a CTA owns one chunk of one row (at most 256 * 8 vectors), everything in registers: 16-byte
+// coalesced loads that are all issued before the first use, max / sum e^x / sum x e^x by warp shuffles, the chunk's
+// Top-K from the K-th largest of 32 group maxima as the bound; the last chunk of a row to arrive merges the row.
+// ================================================================================================================
+template <bool BF16>
+__global__ void __launch_bounds__(HS_ROW_THREADS, 2) quantify_chunk_kernel(const QuantParams p) {
     constexpr int VE = BF16 ? 8 : 4;
     constexpr int VPT = HS_ROW_VPT;
-    extern __shared__ __align__(16) unsigned char s_stage[];   // STAGED: the chunk, HS_ROW_THREADS * VPT vectors
-    __shared__ unsigned long long s_bar;
     __shared__ unsigned long long s_cand[CAND_CAP];
     __shared__ unsigned long long s_top[HS_MAX_TOPK];
     __shared__ unsigned long long s_red[8];
@@ -136,51 +660,22 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, MODE ? 4 : 2) quantify_kernel(
     if (tid < HS_MAX_TOPK) s_top[tid] = 0ull;
     if (tid == 0) s_cnt = 0;
 
-    // ---- the chunk comes on chip: one bulk copy (STAGED) or all loads first ---------------------------
     const unsigned int ninf = BF16 ? 0xff80ff80u : 0xff800000u;
-    uint4 d[STAGED ? 1 : VPT];
-    const uint4* sv = reinterpret_cast<const uint4*>(s_stage);
-    if (STAGED) {
-        const unsigned int bar = smem_u32(&s_bar);
-        if (tid == 0) {
-            mbar_init(bar, 1);
-            mbar_init_fence();
-            const unsigned int bytes = (unsigned int)max(v1 - v0, 0) * 16u;
-            mbar_expect_tx(bar, bytes);
-            if (bytes) bulk_load(smem_u32(s_stage), (const uint4*)(rowp) + v0, bytes, bar);
-        }
-        pdl_launch_dependents();
-        pdl_wait();        // the copy above is in flight; partials and outputs may still be in use upstream
-        __syncthreads();   // the barrier is initialised
-        mbar_wait(bar, 0u, p.err);
-    } else {
+    uint4 d[VPT];
+    pdl_launch_dependents();
+    pdl_wait();
 #pragma unroll
-        for (int j = 0; j < VPT; ++j) {
-            int v = v0 + tid + j * HS_ROW_THREADS;
-            d[STAGED ? 0 : j] = (v < v1) ? __ldcs((const uint4*)(rowp) + v) : make_uint4(ninf, ninf, ninf, ninf);
-        }
-        pdl_launch_dependents();
-        pdl_wait();        // the loads above are in flight; partials and outputs may still be in use upstream
+    for (int j = 0; j < VPT; ++j) {
+        int v = v0 + tid + j * HS_ROW_THREADS;
+        d[j] = (v < v1) ? __ldcs((const uint4*)(rowp) + v) : make_uint4(ninf, ninf, ninf, ninf);
     }
-    // vector j of this thread: from shared memory or from its registers
-    auto vec = [&](int j) -> uint4 {
-        if (STAGED) {
-            const int v = tid + j * HS_ROW_THREADS;
-            return (v0 + v < v1) ? sv[v] : make_uint4(ninf, ninf, ninf, ninf);
-        }
-        return d[STAGED ? 0 : j];
-    };
     // ---- maxima ---------------------------------------------------------------------------
-    // Rolled loops over the vectors need 40 registers instead of 64, so six CTAs share an SM: measured 20 % faster
-    // on launches of many waves, 3 us slower on a launch that is resident at once (the launcher chooses).  The
-    // candidate scan is rolled in both staged variants: few threads run it, mostly from a cold instruction cache.
-    constexpr int UJ = MODE == 2 ? 2 : VPT, UC = MODE != 0 ? 1 : VPT;
-    float vmax[STAGED ? 1 : VPT];
+    float vmax[VPT];
     float tmax = -CUDART_INF_F;
-#pragma unroll UJ
+#pragma unroll
     for (int j = 0; j < VPT; ++j) {
         float x[8];
-        unpack<BF16>(vec(j), x);
+        unpack<BF16>(d[j], x);
         int v = v0 + tid + j * HS_ROW_THREADS;
         if (v == p.nvec - 1) {                       // the row's last vector may run past vocab
 #pragma unroll
@@ -190,16 +685,16 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, MODE ? 4 : 2) quantify_kernel(
         float m = x[0];
 #pragma unroll
         for (int e = 1; e < VE; ++e) m = fmaxf(m, x[e]);
-        if (!STAGED) vmax[STAGED ? 0 : j] = m;
+        vmax[j] = m;
         tmax = fmaxf(tmax, m);
     }
     // ---- sums relative to the thread's own maximum ------------------------------------------
     const float nml = (tmax == -CUDART_INF_F) ? 0.f : -tmax * LOG2E;
     float s = 0.f, u = 0.f;
-#pragma unroll UJ
+#pragma unroll
     for (int j = 0; j < VPT; ++j) {
         float x[8];
-        unpack<BF16>(vec(j), x);
+        unpack<BF16>(d[j], x);
         int v = v0 + tid + j * HS_ROW_THREADS;
         if (v == p.nvec - 1) {
 #pragma unroll
@@ -245,24 +740,17 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, MODE ? 4 : 2) quantify_kernel(
         if (lane == 0) p.part_stats[(size_t)row * p.chunks + chunk] = make_float4(M, St, Ut, 0.f);
     }
     // ---- Top-K of the chunk -------------------------------------------------------------------
-    float tau;
-    {
-        float v = s_gm[lane];
-        int ge = 0;
-#pragma unroll
-        for (int j = 0; j < 32; ++j) ge += (__shfl_sync(HS_FULL_MASK, v, j) >= v);
-        tau = warp_max(ge >= K ? v : -CUDART_INF_F);   // K-th largest group maximum
-    }
+    const float tau = warp_kth_largest(s_gm[lane], K, lane);   // K-th largest group maximum
     if (tmax >= tau && tmax > -CUDART_INF_F) {
-#pragma unroll UC
+#pragma unroll
         for (int j = 0; j < VPT; ++j) {
-            if (STAGED || vmax[STAGED ? 0 : j] >= tau) {
+            if (vmax[j] >= tau) {
                 float x[8];
-                unpack<BF16>(vec(j), x);
+                unpack<BF16>(d[j], x);
                 int base = (v0 + tid + j * HS_ROW_THREADS) * VE;
 #pragma unroll
                 for (int e = 0; e < VE; ++e) {
-                    if (x[e] >= tau && base + e < p.vocab) {
+                    if (x[e] >= tau && x[e] > -CUDART_INF_F && base + e < p.vocab) {
                         int slot = atomicAdd(&s_cnt, 1);
                         if (slot < CAND_CAP) s_cand[slot] = make_key(x[e], base + e);
                     }
@@ -273,17 +761,17 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, MODE ? 4 : 2) quantify_kernel(
     __syncthreads();
     const int ncand = s_cnt;
     if (ncand <= CAND_CAP) {
-        rank_select(s_cand, ncand, K, s_top);
+        rank_select(s_cand, ncand, K, s_top, tid, HS_ROW_THREADS);
     } else {
         // Heavy ties (e.g. a constant row): K rounds of "largest key below the previous one",
         // re-reading the chunk from global memory (cold path).
-        topk_by_rounds<BF16>(rowp, v0, v1, p.vocab, K, s_top, s_red);
+        topk_by_rounds<BF16>(rowp, v0, v1, p.vocab, K, s_top, s_red, tid, HS_ROW_THREADS, 0);
     }
     __syncthreads();
     if (tid < HS_MAX_TOPK)
         p.part_keys[((size_t)row * p.chunks + chunk) * HS_MAX_TOPK + tid] = (tid < K) ? s_top[tid] : 0ull;
 
-    // ---- stage 2: the last chunk of this row merges -----------------------------------------------
+    // ---- the last chunk of this row merges -----------------------------------------------
     // (the CTA's stores are ordered before thread 0's fence by the barrier, the fence before its arrival)
     __syncthreads();
     if (tid == 0) {
@@ -298,7 +786,7 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, MODE ? 4 : 2) quantify_kernel(
         s_cand[t] = __ldcg(&p.part_keys[(size_t)row * p.chunks * HS_MAX_TOPK + t]);
     if (tid < HS_MAX_TOPK) s_top[tid] = 0ull;
     __syncthreads();
-    rank_select(s_cand, nk, K, s_top);
+    rank_select(s_cand, nk, K, s_top, tid, HS_ROW_THREADS);
     __syncthreads();
     if (warp == 0) {
         float m = -CUDART_INF_F, cs = 0.f, cu = 0.f;
@@ -309,195 +797,9 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, MODE ? 4 : 2) quantify_kernel(
         float M = warp_max(m);
         float f = (m == -CUDART_INF_F) ? 0.f : ex2f((m - M) * LOG2E);
         float S = warp_sum(cs * f), U = warp_sum(cu * f);
-        float lse = M + logf(S);
-        float H = lse - U / S;
-        // Top-K entropies: lanes 0..K-1 hold one entry each
-        unsigned long long key = (lane < K) ? s_top[lane] : 0ull;
-        bool valid = key != 0ull;
-        float tv = valid ? key_value(key) : 0.f;
-        float t0 = __shfl_sync(HS_FULL_MASK, tv, 0);
-        float pv = valid ? expf(tv - lse) : 0.f;
-        float itr = warp_sum(valid ? -pv * (tv - lse) : 0.f);
-        float z = valid ? expf(tv - t0) : 0.f;
-        float Z = warp_sum(z);
-        float itk = logf(Z) - warp_sum(valid ? z * (tv - t0) : 0.f) / Z;
-        if (lane < K) {
-            p.out.topk_val[(size_t)row * K + lane] = valid ? tv : -CUDART_INF_F;
-            p.out.topk_idx[(size_t)row * K + lane] = valid ? key_index(key) : -1;
-        }
-        if (lane == 0) {
-            p.out.row_max[row] = M;
-            p.out.row_lse[row] = lse;
-            p.out.h_full[row] = fmaxf(H, 0.f);
-            p.out.i_topk[row] = fmaxf(itk, 0.f);
-            p.out.i_trunc[row] = itr;
-            p.row_cnt[row] = 0;                 // ready for the next launch
-        }
+        finalize_row(p, row, M, S, U, s_top, lane);
+        if (lane == 0) p.row_cnt[row] = 0;                 // ready for the next launch
     }
-    // sequences without any node never reach stage 3: flag them here (first CTA only)
-    if (row == 0) {
-        for (int b = tid; b < p.batch; b += HS_ROW_THREADS)
-            if (p.node_off[b + 1] <= p.node_off[b]) {
-                p.out.status[b] = HS_ERR_BAD_TREE; p.out.pstar_node[b] = 0; p.out.phi_star[b] = 0.f;
-            }
-    }
-    // ---- stage 3: the last row of this tree scores the tree -----------------------------------------
-    __syncthreads();
-    if (tid == 0) {
-        __threadfence();
-        int lo = 0, hi = p.batch;               // largest b with node_off[b] <= row
-        while (hi - lo > 1) {
-            int mid = (lo + hi) >> 1;
-            if (p.node_off[mid] <= row) lo = mid; else hi = mid;
-        }
-        int n = p.node_off[lo + 1] - p.node_off[lo];
-        int last = (atomicAdd(&p.tree_cnt[lo], 1) == n - 1);
-        if (last) p.tree_cnt[lo] = 0;
-        s_flag = last ? lo : -1;
-        __threadfence();
-    }
-    __syncthreads();
-    const int b = s_flag;
-    if (b < 0) return;
-    tree_scores(p, b, (float*)s_cand, (int*)(s_cand + 256));
-}
-
-// One CTA, n <= HS_MAX_NODES nodes.  s_f: 3*128 floats, s_i: 2*128 ints of shared memory.
-__device__ void tree_scores(const QuantParams& p, int b, float* s_f, int* s_i) {
-    __shared__ unsigned long long s_best[8];
-    __shared__ int s_maxd[8];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int base = p.node_off[b];
-    const int n = p.node_off[b + 1] - base;
-    float* s_logc = s_f;
-    float* s_I = s_f + HS_MAX_NODES;
-    float* s_phi = s_f + 2 * HS_MAX_NODES;
-    int* s_par = s_i;
-    // validation
-    int bad = (n > HS_MAX_NODES);
-    int par = -1, tok = 0;
-    if (!bad && tid < n) {
-        par = p.parent[base + tid];
-        tok = p.token[base + tid];
-        if (tid == 0) bad = (par != -1);
-        else bad = (par < 0 || par >= tid || tok < 0 || tok >= p.vocab);
-    }
-    bad = __syncthreads_or(bad);
-    if (bad) {
-        for (int i = tid; i < n; i += blockDim.x) {
-            p.out.logc[base + i] = 0.f; p.out.score[base + i] = 0.f; p.out.phi[base + i] = 0.f;
-            p.out.depth[base + i] = 0;
-        }
-        if (tid == 0) { p.out.status[b] = HS_ERR_BAD_TREE; p.out.pstar_node[b] = 0; p.out.phi_star[b] = 0.f; }
-        return;
-    }
-    if (tid < n) {
-        float lc = 0.f;
-        if (tid > 0) {
-            size_t off = (size_t)(base + par) * p.row_stride + tok;
-            float lv = p.is_bf16 ? __bfloat162float(((const __nv_bfloat16*)p.logits)[off])
-                                 : ((const float*)p.logits)[off];
-            lc = lv - __ldcg(&p.out.row_lse[base + par]);
-        }
-        s_logc[tid] = lc;
-        s_I[tid] = __ldcg(p.entropy_mode == 0 ? &p.out.i_topk[base + tid] : &p.out.i_trunc[base + tid]);
-        s_par[tid] = par;
-    }
-    __syncthreads();
-    float S = 0.f, Phi = 0.f;
-    int dep = 0;
-    if (tid < n) {
-        int a = tid;
-        while (a > 0) {
-            int pa = s_par[a];
-            S += s_logc[a];
-            Phi += s_I[pa];
-            a = pa;
-            ++dep;
-        }
-        if (p.phi_mode == 1) Phi += s_I[tid];
-        s_phi[tid] = Phi;
-        p.out.logc[base + tid] = s_logc[tid];
-        p.out.score[base + tid] = S;
-        p.out.phi[base + tid] = Phi;
-        p.out.depth[base + tid] = dep;
-    }
-    // deepest level, then P* among the nodes of depth min(d_base, deepest)
-    int md = dep;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) md = max(md, __shfl_xor_sync(HS_FULL_MASK, md, o));
-    if (lane == 0) s_maxd[warp] = md;
-    __syncthreads();
-    md = s_maxd[0];
-    for (int w = 1; w < 8; ++w) md = max(md, s_maxd[w]);
-    const int t_eval = min(p.d_base, md);
-    unsigned long long key = 0ull;
-    if (tid < n && dep == t_eval) key = make_key(p.pstar_mode == 0 ? s_logc[tid] : S, tid);
-    key = warp_max_u64(key);
-    if (lane == 0) s_best[warp] = key;
-    __syncthreads();
-    if (tid == 0) {
-        unsigned long long best = s_best[0];
-        for (int w = 1; w < 8; ++w) best = s_best[w] > best ? s_best[w] : best;
-        int node = key_index(best);
-        p.out.pstar_node[b] = node;
-        p.out.phi_star[b] = s_phi[node];
-        p.out.status[b] = HS_OK;
-    }
-}
-
-hs_status hs_launch_quantify(hs_ctx* ctx, const hs_tree_batch* tree, const void* logits, hs_dtype dtype,
-                             int64_t row_stride, int32_t vocab, const hs_policy* policy,
-                             const hs_quant_out* out, cudaStream_t stream) {
-    QuantParams p;
-    const int ve = hs_vec_elems(dtype);
-    p.logits = logits;
-    p.row_stride = row_stride;
-    p.vocab = vocab;
-    p.nvec = (vocab + ve - 1) / ve;
-    p.chunks = hs_row_chunks(vocab, dtype);
-    if (p.chunks * HS_MAX_TOPK > CAND_CAP || p.chunks > 32) return HS_ERR_SHAPE;
-    p.chunk_vecs = (p.nvec + p.chunks - 1) / p.chunks;
-    p.rows = tree->n_nodes_total;
-    p.batch = tree->batch;
-    p.node_off = tree->node_off;
-    p.parent = tree->parent;
-    p.token = tree->token;
-    p.out = *out;
-    size_t stats_bytes = hs_align_up((size_t)p.rows * p.chunks * sizeof(float4), 256);
-    size_t keys_bytes = (size_t)p.rows * p.chunks * HS_MAX_TOPK * sizeof(unsigned long long);
-    if (stats_bytes + keys_bytes > ctx->scratch_bytes) return HS_ERR_WORKSPACE;
-    p.part_stats = (float4*)ctx->scratch;
-    p.part_keys = (unsigned long long*)(ctx->scratch + stats_bytes);
-    p.row_cnt = ctx->counters + HS_CNT_QUANT_ROW;
-    p.tree_cnt = ctx->counters + HS_CNT_QUANT_TREE;
-    p.K = policy->top_k;
-    p.d_base = policy->d_base;
-    p.phi_mode = policy->phi_mode;
-    p.pstar_mode = policy->pstar_mode;
-    p.entropy_mode = policy->entropy_mode;
-    p.is_bf16 = dtype == HS_BF16;
-    p.err = ctx->counters + HS_CNT_ERROR;
-    dim3 grid(p.chunks, p.rows);
-    // the bulk copy wants 16-byte aligned rows
-    const size_t esz = dtype == HS_BF16 ? 2 : 4;
-    const bool staged = ((uintptr_t)logits % 16 == 0) && ((size_t)row_stride * esz % 16 == 0);
-    const size_t stage_bytes = (size_t)HS_ROW_THREADS * HS_ROW_VPT * 16;
-    const bool many_waves = (long long)p.chunks * p.rows > 4ll * ctx->sm_count;
-    cudaError_t e;
-    if (staged && many_waves)
-        e = dtype == HS_BF16
-            ? hs_launch(quantify_kernel<true, 2>, grid, dim3(HS_ROW_THREADS), stage_bytes, stream, ctx->pdl, dim3(1, 1, 1), p)
-            : hs_launch(quantify_kernel<false, 2>, grid, dim3(HS_ROW_THREADS), stage_bytes, stream, ctx->pdl, dim3(1, 1, 1), p);
-    else if (staged)
-        e = dtype == HS_BF16
-            ? hs_launch(quantify_kernel<true, 1>, grid, dim3(HS_ROW_THREADS), stage_bytes, stream, ctx->pdl, dim3(1, 1, 1), p)
-            : hs_launch(quantify_kernel<false, 1>, grid, dim3(HS_ROW_THREADS), stage_bytes, stream, ctx->pdl, dim3(1, 1, 1), p);
-    else
-        e = dtype == HS_BF16
-            ? hs_launch(quantify_kernel<true, 0>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p)
-            : hs_launch(quantify_kernel<false, 0>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p);
-    return e == cudaSuccess ? HS_OK : HS_ERR_CUDA;
 }
 
 // ---- hs_entropy_quantify_static: the same pass without any allocated workspace -------------------------------
@@ -508,7 +810,7 @@ hs_status hs_launch_quantify(hs_ctx* ctx, const hs_tree_batch* tree, const void*
 // in one fixed array that is part of the library image, so every GPU that loads the library carries
 // HS_STATIC_SCRATCH_BYTES of it until the process exits.
 #define HS_STATIC_MAX_CHUNKS 16
-#define HS_STATIC_COUNTER_BYTES 2048    // (HS_STATIC_MAX_ROWS + HS_STATIC_MAX_BATCH) ints, rounded up
+#define HS_STATIC_COUNTER_BYTES 2048    // HS_STATIC_MAX_ROWS ints (one arrival counter per row), rounded up
 #define HS_STATIC_STATS_BYTES (HS_STATIC_MAX_ROWS * HS_STATIC_MAX_CHUNKS * 16)
 #define HS_STATIC_KEYS_BYTES (HS_STATIC_MAX_ROWS * HS_STATIC_MAX_CHUNKS * HS_MAX_TOPK * 8)
 #define HS_STATIC_SCRATCH_BYTES (HS_STATIC_COUNTER_BYTES + HS_STATIC_STATS_BYTES + HS_STATIC_KEYS_BYTES)
@@ -557,33 +859,18 @@ extern "C" hs_status hs_entropy_quantify_static(const hs_tree_batch* tree, const
     }
 
     QuantParams p;
-    p.logits = draft_logits;
-    p.row_stride = row_stride;
-    p.vocab = vocab;
-    p.nvec = (vocab + ve - 1) / ve;
+    fill_common(p, tree, draft_logits, dtype, row_stride, vocab, policy, out);
     p.chunks = chunks;
     p.chunk_vecs = (p.nvec + p.chunks - 1) / p.chunks;
-    p.rows = tree->n_nodes_total;
-    p.batch = tree->batch;
-    p.node_off = tree->node_off;
-    p.parent = tree->parent;
-    p.token = tree->token;
-    p.out = *out;
     p.row_cnt = (int*)base;
-    p.tree_cnt = (int*)base + HS_STATIC_MAX_ROWS;
     p.part_stats = (float4*)(base + HS_STATIC_COUNTER_BYTES);
     p.part_keys = (unsigned long long*)(base + HS_STATIC_COUNTER_BYTES + HS_STATIC_STATS_BYTES);
-    p.K = policy->top_k;
-    p.d_base = policy->d_base;
-    p.phi_mode = policy->phi_mode;
-    p.pstar_mode = policy->pstar_mode;
-    p.entropy_mode = policy->entropy_mode;
-    p.is_bf16 = dtype == HS_BF16;
     // The array keeps whatever the previous call left: the arrival counters must start at zero.
     HS_CUDA_OK(cudaMemsetAsync(base, 0, HS_STATIC_COUNTER_BYTES, stream));
     dim3 grid(p.chunks, p.rows);
-    p.err = nullptr;       // (the register variant has no bounded wait)
-    if (dtype == HS_BF16) quantify_kernel<true, 0><<<grid, HS_ROW_THREADS, 0, stream>>>(p);
-    else quantify_kernel<false, 0><<<grid, HS_ROW_THREADS, 0, stream>>>(p);
+    if (dtype == HS_BF16) quantify_chunk_kernel<true><<<grid, HS_ROW_THREADS, 0, stream>>>(p);
+    else quantify_chunk_kernel<false><<<grid, HS_ROW_THREADS, 0, stream>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return HS_ERR_CUDA;
+    tree_scores_kernel<<<p.batch, HS_MAX_NODES, 0, stream>>>(p);      // (needs no scratch)
     return cudaGetLastError() == cudaSuccess ? HS_OK : HS_ERR_CUDA;
 }

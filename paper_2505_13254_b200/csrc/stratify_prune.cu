@@ -3,8 +3,10 @@
 // Entropy bin -> (d', N') (Sec. 4.2-4.3), Top-N' reranking by path confidence (Sec. 2.2), then the
 // surviving nodes are compacted with warp ballots and a prefix sum over the four warps, parents are
 // re-indexed and each kept node gets its ancestor-or-self bit mask (the tree-attention mask).
-// The CSR offset of a sequence is the sum of the kept counts of all earlier sequences; every CTA
-// recomputes those counts itself, so no CTA waits for another.
+// The CSR offset of a sequence is the sum of the kept counts of all earlier sequences.  Small batches:
+// every CTA recomputes those counts itself, so no CTA waits for another and the call is one launch.
+// Larger batches: a first launch counts the kept nodes of every sequence once (one warp each), the
+// second sums the counts ahead of its sequence (B integers instead of B trees per CTA).
 #include "hs_common.cuh"
 #include "hs_layout.h"
 #include "hs_ptx.cuh"
@@ -18,6 +20,7 @@ struct PruneParams {
     const int* depth;
     const int* qstatus;
     hs_pruned_tree out;
+    int counted;           // out.n_keep was filled by prune_count_kernel
     float th[7];
     int d_base, alpha, n_default, gamma_pct[3];
 };
@@ -46,6 +49,27 @@ __device__ __forceinline__ int kept_count(const PruneParams& p, int b) {
     return max(0, min(np, elig));
 }
 
+// one warp per sequence: its kept count -> out.n_keep[b]
+__global__ void __launch_bounds__(128) prune_count_kernel(const PruneParams p) {
+    const int lane = threadIdx.x & 31;
+    const int b = blockIdx.x * 4 + (threadIdx.x >> 5);
+    pdl_launch_dependents();
+    pdl_wait();
+    if (b >= p.batch) return;
+    int cnt = 0;
+    if (p.qstatus[b] == 0) {
+        int bin, dp, np;
+        policy_lookup(p, p.phi_star[b], bin, dp, np);
+        const int lo = p.node_off[b], hi = min(p.node_off[b + 1], lo + HS_MAX_NODES);
+        int elig = 0;
+        for (int i = lo + lane; i < hi; i += 32) elig += (p.depth[i] <= dp);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) elig += __shfl_xor_sync(HS_FULL_MASK, elig, o);
+        cnt = max(0, min(np, elig));
+    }
+    if (lane == 0) p.out.n_keep[b] = cnt;
+}
+
 __global__ void __launch_bounds__(HS_MAX_NODES) stratify_prune_kernel(const PruneParams p) {
     __shared__ float s_S[HS_MAX_NODES];
     __shared__ int s_elig[HS_MAX_NODES];
@@ -62,7 +86,11 @@ __global__ void __launch_bounds__(HS_MAX_NODES) stratify_prune_kernel(const Prun
 
     // offset of this sequence in the compacted arrays
     int part = 0;
-    for (int bb = tid; bb < b; bb += HS_MAX_NODES) part += kept_count(p, bb);
+    if (p.counted) {
+        for (int bb = tid; bb < b; bb += HS_MAX_NODES) part += p.out.n_keep[bb];
+    } else {
+        for (int bb = tid; bb < b; bb += HS_MAX_NODES) part += kept_count(p, bb);
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(HS_FULL_MASK, part, o);
     if (lane == 0) s_warp[warp] = part;
@@ -150,6 +178,10 @@ hs_status hs_launch_stratify_prune(hs_ctx* ctx, const hs_tree_batch* tree, const
     p.alpha = policy->alpha;
     p.n_default = policy->n_default;
     for (int i = 0; i < 3; ++i) p.gamma_pct[i] = policy->gamma_pct[i];
+    p.counted = p.batch > 32;
+    if (p.counted &&
+        hs_launch(prune_count_kernel, dim3((p.batch + 3) / 4), dim3(128), 0, stream, ctx->pdl, dim3(1, 1, 1), p) != cudaSuccess)
+        return HS_ERR_CUDA;
     return hs_launch(stratify_prune_kernel, dim3(p.batch), dim3(HS_MAX_NODES), 0, stream, ctx->pdl, dim3(1, 1, 1), p) ==
                    cudaSuccess ? HS_OK : HS_ERR_CUDA;
 }

@@ -43,7 +43,7 @@ struct AttnParams {
     const int* status;
     const int* node_off;
     const int* kv_off;
-    int batch, hq, hkv, G, layout, nsplit, head_first;
+    int batch, hq, hkv, G, layout, nsplit, head_first, prefetch;
     float scale_log2;
     int* err;
 };
@@ -151,7 +151,8 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         mbar_init(bar_sr, UM_ROWS_THREADS);              // S of a tile is in registers: its buffer may take the next S
         mbar_init(bar_sr + 8, UM_ROWS_THREADS);
         mbar_init_fence();
-        for (int i = 0; i < pre; ++i) { issue_kv(i, false); issue_kv(i, true); }
+        if (p.prefetch)                                  // the caller vouches for the cache: tiles requested ahead of the wait
+            for (int i = 0; i < pre; ++i) { issue_kv(i, false); issue_kv(i, true); }
     }
     if (warp == 0) {
         tmem_alloc(tslot, UM_TMEM_COLS);
@@ -159,6 +160,8 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
     }
     pdl_launch_dependents();
     pdl_wait();                                      // the pruned tree, q, k_tree, v_tree come from upstream
+    if (tid == 0 && !p.prefetch)
+        for (int i = 0; i < pre; ++i) { issue_kv(i, false); issue_kv(i, true); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -642,14 +645,13 @@ static void query_cluster_caps(Kernel kernel, int threads, size_t smem, int sm_c
 hs_status hs_launch_attention(hs_ctx* ctx, const hs_pruned_tree* pruned, const hs_attn_desc* d, const void* q,
                               const void* k_tree, const void* v_tree, const void* k_cache, const void* v_cache,
                               void* out, float* lse_out, cudaStream_t stream) {
-    static bool attr_set = false;
-    static int cap_umma[ATT_MAX_SPLIT + 1];          // CTAs that run at once in clusters of s
-    if (!attr_set) {
+    int* cap_umma = ctx->attn_cap;                   // CTAs that run at once in clusters of s (per device = per context)
+    if (!ctx->attn_ready) {
         if (cudaFuncSetAttribute(tree_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, UM_SMEM_BYTES) !=
             cudaSuccess)
             return HS_ERR_CUDA;
         query_cluster_caps(tree_attn_umma_kernel, UM_THREADS, UM_SMEM_BYTES, ctx->sm_count, cap_umma);
-        attr_set = true;
+        ctx->attn_ready = true;
     }
     AttnParams p;
     p.q = (const __nv_bfloat16*)q;
@@ -672,6 +674,7 @@ hs_status hs_launch_attention(hs_ctx* ctx, const hs_pruned_tree* pruned, const h
     p.head_first = d->kv_head_stride > d->kv_token_stride;
     p.scale_log2 = d->sm_scale * LOG2E;
     p.err = ctx->counters + HS_CNT_ERROR;
+    p.prefetch = (ctx->prefetch & HS_PREFETCH_KV) != 0;
     const int pairs = d->batch * d->hkv;
     const int mblocks = (p.G * d->max_nodes + ATT_BM - 1) / ATT_BM;
     const int prefix_tiles = (d->max_kv_len + ATT_BN - 1) / ATT_BN;

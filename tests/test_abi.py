@@ -27,7 +27,7 @@ def test_status_strings_and_workspace_size_need_no_gpu():
     L = binding.lib()
     assert L.hs_status_string(0) == b"ok"
     assert L.hs_status_string(7) == b"malformed tree"
-    assert binding.hs_workspace_bytes(1, 60, 128256, 32, 8) >= 64 << 20
+    assert 256 << 10 < binding.hs_workspace_bytes(1, 60, 128256, 32, 8) < 4 << 20     # counters + chunk partials only
     assert binding.hs_workspace_bytes(0, 60, 128256, 32, 8) == 0
 
 

@@ -32,3 +32,13 @@ def test_streams_differ():
     assert a != philox.uniform(8, 0, 0, 5, 0)
     assert a != philox.uniform(7 + (1 << 32), 0, 0, 5, 0)     # high key word is used
     assert a == philox.uniform(7, 0, 0, 5, 0)
+
+
+def test_offset_high_word_selects_another_stream():
+    """Counter convention of the acceptance step: (offset low word, b, node, stream + 2 * offset high word)."""
+    seed = 0x0123456789ABCDEF
+    key = (seed & 0xFFFFFFFF, seed >> 32)
+    for off, b, node, stream in ((0, 0, 0, 0), (7, 3, 5, 1), ((9 << 32) + 7, 3, 5, 1), ((1 << 63) - 1, 4095, 127, 0)):
+        words = philox.philox4x32_10((off & 0xFFFFFFFF, b, node, stream + 2 * (off >> 32)), key)
+        assert philox.uniform(seed, off, b, node, stream) == (words[0] >> 8) * 2.0 ** -24
+    assert philox.uniform(seed, 7, 3, 5, 1) != philox.uniform(seed, (1 << 32) + 7, 3, 5, 1)

@@ -34,12 +34,14 @@ def test_static_scratch_matches_the_workspace_path_twice_in_a_row():
              (synth.CONFIGS["c1_tiny"].scaled(kv_len=(8, 8)), "c1_tiny", 72)]
     for cfg, base, seed in cases:                         # bf16 ragged batch, then an fp32 tree
         policy = pu.policy_for(cfg, base)
-        db = gstep.upload(synth.make_batch(cfg, seed, with_attention=False))
+        batch, res = pu.oracle_case(cfg, policy, seed, attention="none")
+        db = gstep.upload(batch)
         want = hb.hs_entropy_quantify(ctx, db.tree, db.draft, policy)
         got = hb.hs_entropy_quantify_static(db.tree, db.draft, policy)
         torch.cuda.synchronize()
         assert int(got.status.abs().sum()) == 0
         _compare(got, want)
+        pu.check_quant(got, batch, res, policy["top_k"])     # and against the CPU oracle, like every other path
     ctx.close()
 
 
