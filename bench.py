@@ -27,6 +27,26 @@ import numpy as np  # noqa: E402
 METRIC = "verified_draft_trees_per_second"
 UNIT = "trees/s"
 L2_BYTES = 126 << 20
+NOMINAL_HBM_GBS = 8000.0          # the part's nominal HBM3e bandwidth
+NOMINAL_BF16_TFLOPS = 2250.0      # nominal dense bf16
+
+
+def workload_config(cfg):
+    """The workload's description, identical in both arms of the benchmark."""
+    return {"workload": cfg.name, "batch_per_gpu": cfg.batch, "tree_nodes": list(cfg.n_nodes), "vocab": cfg.vocab,
+            "logits_dtype": cfg.logits_dtype, "kv_len": list(cfg.kv_len), "hq": cfg.hq, "hkv": cfg.hkv,
+            "head_dim": cfg.head_dim, "attention_layers_per_step": 1, "accept": cfg.accept}
+
+
+def oracle_threads():
+    """Threads the numpy oracle can use: its loops are single-threaded python; only BLAS calls (the
+    matrix-vector products of the attention) may use the BLAS pool."""
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([int(i.get("num_threads", 1)) for i in threadpool_info()] or [1])
+    except Exception:
+        n = 1
+    return n
 
 
 def load_policy(cfg, synth):
@@ -38,7 +58,7 @@ def ncu_traffic(kernel, workload):
     """DRAM bytes per launch of `kernel` from the committed ncu capture, or None if there is none or the
     kernel's source has changed since the counters were taken."""
     import hashlib
-    path = os.path.join(ROOT, "paper_2505_13254_b200", "ncu_traffic.json")
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
     if not os.path.exists(path):
         return None
     ent = json.load(open(path)).get(kernel, {}).get(workload)
@@ -151,15 +171,15 @@ def run_reference(args, cfg, synth):
             times.append(dt)
     total = sum(times)
     value = cfg.batch * len(times) / total
-    cores = os.cpu_count()
+    cores = oracle_threads()
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": {"workload": cfg.name, "batch": cfg.batch, "vocab": cfg.vocab,
-                                            "kv_len": cfg.kv_len[1], "hq": cfg.hq, "hkv": cfg.hkv},
+            "data": "synthetic", "config": workload_config(cfg),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                              "sample": "each step = the whole batch through the numpy fp64 oracle (all logits rows, "
-                                       "all kept-node attention pairs of one layer); numpy/BLAS threads as configured"},
+                                       "all kept-node attention pairs of one layer); python loops on one core, BLAS "
+                                       "calls on `cores` threads (host has %d cores)" % (os.cpu_count() or 0)},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -174,6 +194,9 @@ def main():
     ap.add_argument("--workload", default="c2_8b")
     ap.add_argument("--rotate", type=int, default=0, help="distinct input copies (0 = enough to exceed 2x L2)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--prefetch", default="all", choices=["none", "kv", "all"],
+                    help="inputs the kernels may fetch before their dependency wait (hs_set_prefetch): the benchmark's "
+                         "logits and KV cache are resident and never written by the kernel ahead of a call")
     ap.add_argument("--accept", default=None, choices=["greedy", "rejection", "mixed", "deterministic", "mixed3"],
                     help="acceptance mode(s) of the sequences instead of the workload's own")
     args = ap.parse_args()
@@ -215,6 +238,7 @@ def main():
         sets.append(c)
     ws = hb.hs_workspace_bytes(cfg.batch, db0.tree.n_nodes_total, cfg.vocab, cfg.hq, cfg.hkv)
     ctx = hb.Context(local, ws)
+    hb.hs_set_prefetch(ctx, {"none": 0, "kv": hb.HS_PREFETCH_KV, "all": hb.HS_PREFETCH_KV | hb.HS_PREFETCH_LOGITS}[args.prefetch])
     st = gstep.VerifyStep(ctx, db0, policy)
 
     def barrier():
@@ -331,7 +355,7 @@ def main():
     attn_bytes = 2 * (L + nk) * cfg.hkv * cfg.head_dim * 2 + 2 * nk * cfg.hq * cfg.head_dim * 2
     accept_bytes = nk * cfg.vocab * esz
     kern = {
-        "quantify": {"bytes": quant_bytes, "us": call_us["quantify"], "launches_per_step": 1},
+        "quantify": {"bytes": quant_bytes, "us": call_us["quantify"], "launches_per_step": 2},
         "attention": {"bytes": attn_bytes, "us": call_us["attention"], "launches_per_step": 1},
         "accept_path": {"bytes": accept_bytes, "us": call_us["accept_path"],
                         "launches_per_step": 2 if db0.any_sampling else 1},
@@ -340,29 +364,31 @@ def main():
     for k in kern.values():
         k["gbs"] = k["bytes"] / (k["us"] * 1e-6) / 1e9 if k["us"] > 0 else None
         k["frac_of_%s_hbm" % peak_kind] = k["gbs"] / peak if k["gbs"] else None
-    traffic = ncu_traffic("quantify_kernel", cfg.name)
+        k["frac_of_nominal_hbm"] = k["gbs"] / NOMINAL_HBM_GBS if k["gbs"] else None
+    traffic = ncu_traffic("quantify_stream_kernel", cfg.name)
     achieved = kern["quantify"]["gbs"]
     line = {
         "metric": METRIC, "value": whole_job_value(world, cfg.batch, args.steps, ms), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": cfg.name, "batch_per_gpu": cfg.batch, "tree_nodes": n_rows, "kept_nodes": nk,
-                   "vocab": cfg.vocab, "logits_dtype": cfg.logits_dtype, "kv_len": cfg.kv_len[1], "hq": cfg.hq,
-                   "hkv": cfg.hkv, "head_dim": cfg.head_dim, "attention_layers_per_step": 1,
-                   "accept": cfg.accept, "parallelism": "replicas" if world > 1 else "single",
-                   "l2": "inputs rotate through %d distinct device copies, %.0f MB in total (L2 = 126 MB)"
-                         % (R, R * per_set / 1e6)},
+        "config": workload_config(cfg),
+        "run": {"tree_nodes_total": n_rows, "kept_nodes_total": nk, "parallelism": "replicas" if world > 1 else "single",
+                "prefetch": args.prefetch,
+                "l2": "inputs rotate through %d distinct device copies, %.0f MB in total (L2 = 126 MB)"
+                      % (R, R * per_set / 1e6)},
         "clocks": clocks,
         "e2e": {"value": world * cfg.batch * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": 1e3 * e2e_s / e2e_steps,
                 "how": "every step copies all inputs from pinned host memory and reads its results back; the copies of "
                        "step n + 1 overlap the kernels of step n (two staging buffers, two streams)"},
-        "gpu_launches": (5 if db0.any_sampling else 4) * args.steps,
-        "roofline": {"kernel": "quantify_kernel (hs_entropy_quantify, one launch per step)", "bound": "hbm",
+        "gpu_launches": (6 if db0.any_sampling else 5) * args.steps,
+        "roofline": {"kernel": "quantify_stream_kernel (hs_entropy_quantify: this kernel + the tree stage)", "bound": "hbm",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "frac_of_nominal": achieved / NOMINAL_HBM_GBS,
                      "peak_kind": peak_kind + " (burst copy figure)", "traffic": traffic,
                      "algorithmic_bytes_per_launch": quant_bytes,
-                     "how": "CUDA events around K back-to-back graph-replayed launches of this call alone, inputs rotating"},
+                     "how": "CUDA events around K back-to-back graph-replayed calls of hs_entropy_quantify alone (both of its "
+                            "launches in the duration), inputs rotating"},
         "calls": kern,
         "device_error_word": dev_err,
     }
@@ -376,14 +402,17 @@ def main():
     if attn_flops / (tf_peak * 1e12) > attn_bytes / (peak * 1e9):      # the tensor pipe is the longer leg
         line["roofline_attention"] = {"kernel": "tree_attn_umma_kernel (hs_tree_verify_attention, one launch per step)",
                                       "bound": "tensor", "achieved": a_tflops, "peak": tf_peak, "unit": "TFLOP/s",
-                                      "frac": a_tflops / tf_peak, "peak_kind": peak_kind + " (dense bf16 burst figure)",
+                                      "frac": a_tflops / tf_peak, "frac_of_nominal": a_tflops / NOMINAL_BF16_TFLOPS,
+                                      "peak_kind": peak_kind + " (dense bf16 burst figure)",
                                       "traffic": ncu_traffic("tree_attn_umma_kernel", cfg.name),
                                       "algorithmic_flops_per_launch": attn_flops,
                                       "algorithmic_bytes_per_launch": attn_bytes}
     else:
         line["roofline_attention"] = {"kernel": "tree_attn_umma_kernel (hs_tree_verify_attention, one launch per step)",
                                       "bound": "hbm", "achieved": a_gbs, "peak": peak, "unit": "GB/s",
-                                      "frac": a_gbs / peak if a_gbs else None, "peak_kind": peak_kind + " (burst copy figure)",
+                                      "frac": a_gbs / peak if a_gbs else None,
+                                      "frac_of_nominal": a_gbs / NOMINAL_HBM_GBS if a_gbs else None,
+                                      "peak_kind": peak_kind + " (burst copy figure)",
                                       "traffic": ncu_traffic("tree_attn_umma_kernel", cfg.name),
                                       "algorithmic_bytes_per_launch": attn_bytes,
                                       "algorithmic_flops_per_launch": attn_flops}
@@ -392,7 +421,7 @@ def main():
         nrep = 5
         t = sum(oracle_sample(synth.make_batch(cfg, rank_seed(rank) + 1000 * i) if i else batch, policy, ostep)
                 for i in range(nrep))
-        line["cpu_baseline"] = {"value": nrep * cfg.batch / t, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+        line["cpu_baseline"] = {"value": nrep * cfg.batch / t, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
                                 "sample": "%d batches of this workload (seeds differ) once each through the numpy fp64 "
                                           "oracle: all logits rows, all kept-node attention pairs of one layer (%.1f s)"
                                           % (nrep, t)}

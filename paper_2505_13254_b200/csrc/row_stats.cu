@@ -43,7 +43,10 @@ struct QuantParams {
     int nvec;        // 16-byte vectors per row, the last one may be partial
     int chunks;      // chunk kernel: CTAs per row
     int chunk_vecs;  // chunk kernel: vectors per chunk
-    int per;         // stream kernel: vectors per CTA share
+    int per;         // stream kernel: vectors per share
+    int split;       // stream kernel: shares per row (row-split geometry), 0 = byte-balanced stream
+    int extra;       // stream kernel, row split: the first `extra` rows have one share more
+    int nslots;      // stream kernel: item slots in shared memory
     int rows;
     int batch;
     const int* node_off;
@@ -174,40 +177,86 @@ __device__ __forceinline__ float warp_kth_largest(float v, int K, int lane) {
 // ================================================================================================================
 // The streaming kernel
 // ================================================================================================================
+// Geometry of the shares.  split == 0 ("stream"): the rows form one stream of rows * nvec vectors, share c is
+// [c * per, (c + 1) * per), a share may hold several rows and a row may lie in several shares.  split == S > 0 ("row
+// split", for launches with at most one row per SM): the first `extra` rows are cut into S + 1 equal parts, the
+// others into S, one share per part, so that every share is a single row segment.  split < 0 ("whole rows", for
+// launches with many rows per SM): share c of `extra` shares holds the rows [c * rows / extra, (c + 1) * rows / extra).
+struct Share {
+    long long g0, g1;
+};
+__device__ __forceinline__ void shares_of_row(const QuantParams& p, int row, int& c_first, int& nseg) {
+    if (p.split < 0) {
+        c_first = 0; nseg = 1;
+    } else if (p.split) {
+        if (row < p.extra) { c_first = row * (p.split + 1); nseg = p.split + 1; }
+        else { c_first = p.extra * (p.split + 1) + (row - p.extra) * p.split; nseg = p.split; }
+    } else {
+        const long long r0 = (long long)row * p.nvec;
+        c_first = (int)(r0 / p.per);
+        nseg = (int)((r0 + p.nvec - 1) / p.per) - c_first + 1;
+    }
+}
+__device__ __forceinline__ Share share_of(const QuantParams& p, int c) {
+    Share sh;
+    if (p.split < 0) {
+        sh.g0 = ((long long)c * p.rows / p.extra) * p.nvec;
+        sh.g1 = ((long long)(c + 1) * p.rows / p.extra) * p.nvec;
+    } else if (p.split) {
+        const int wide = p.extra * (p.split + 1);           // shares of the rows with S + 1 parts
+        const int parts = c < wide ? p.split + 1 : p.split;
+        const int row = c < wide ? c / parts : p.extra + (c - wide) / parts;
+        const int part = c < wide ? c - row * parts : (c - wide) - (row - p.extra) * parts;
+        const int pv = (p.nvec + parts - 1) / parts;
+        sh.g0 = (long long)row * p.nvec + min(part * pv, p.nvec);
+        sh.g1 = (long long)row * p.nvec + min((part + 1) * pv, p.nvec);
+    } else {
+        sh.g0 = (long long)c * p.per;
+        sh.g1 = min(sh.g0 + (long long)p.per, (long long)p.rows * p.nvec);
+    }
+    return sh;
+}
+// partial slot of share c for `row`: stream mode has two per share (the leading one for a row that began in an
+// earlier share), row-split mode one
+__device__ __forceinline__ int partial_slot(const QuantParams& p, int row, int c) {
+    if (p.split) return c;
+    return 2 * c + ((long long)row * p.nvec < (long long)c * p.per ? 0 : 1);
+}
+
 template <bool BF16>
 __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const QuantParams p) {
     constexpr int VE = BF16 ? 8 : 4;
+    constexpr int NW = QS_CONSUMERS / 32;
     extern __shared__ __align__(128) unsigned char s_dyn[];
     __shared__ unsigned long long s_full[QS_SLOTS], s_empty[QS_SLOTS];
     __shared__ unsigned long long s_list[CAND_CAP];
-    __shared__ unsigned long long s_top[HS_MAX_TOPK];
-    __shared__ unsigned long long s_red[QS_CONSUMERS / 32];
+    __shared__ unsigned long long s_top[2][HS_MAX_TOPK];   // (two copies: a finished row is written out by warp 0
+    __shared__ unsigned long long s_red[NW];               //  while the other warps read the next one)
     __shared__ float s_gm[32];
-    __shared__ float s_wstat[QS_CONSUMERS / 32][3];
+    __shared__ float s_wstat[2][NW][3];
     __shared__ int s_cnt;
     __shared__ int s_flag;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned int slots0 = (smem_u32(s_dyn) + 127u) & ~127u;
     const unsigned char* slots_gen = s_dyn + (slots0 - smem_u32(s_dyn));
-    const long long total = (long long)p.rows * p.nvec;
-    const long long g0 = (long long)blockIdx.x * p.per;
-    const long long g1 = min(g0 + (long long)p.per, total);
+    const Share sh = share_of(p, blockIdx.x);
+    const long long g0 = sh.g0, g1 = sh.g1;
     const size_t esz = BF16 ? 2 : 4;
+    const int nslots = p.nslots;
 
     if (tid == 0) {
-        for (int s = 0; s < QS_SLOTS; ++s) {
+        for (int s = 0; s < nslots; ++s) {
             mbar_init(smem_u32(&s_full[s]), 1);
-            mbar_init(smem_u32(&s_empty[s]), QS_CONSUMERS / 32);
+            mbar_init(smem_u32(&s_empty[s]), NW);
         }
         mbar_init_fence();
         s_cnt = 0;
     }
-    if (tid < HS_MAX_TOPK) s_top[tid] = 0ull;
     __syncthreads();
     pdl_launch_dependents();
 
-    if (warp == QS_CONSUMERS / 32) {
+    if (warp == NW) {
         // ---- producer: one lane walks the share item by item ----------------------------------------------------
         if (lane == 0) {
             long long g = g0;
@@ -218,10 +267,10 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
                 const int row = (int)(g / p.nvec);
                 const int v = (int)(g - (long long)row * p.nvec);
                 const int len = (int)min((long long)min(QS_ITEM_VECS, p.nvec - v), g1 - g);
-                const int slot = it % QS_SLOTS;
-                if (it >= QS_SLOTS) {
+                const int slot = it % nslots;
+                if (it >= nslots) {
                     if (!waited) { pdl_wait(); waited = true; }     // (nothing of this kernel is written by the producer)
-                    mbar_wait(smem_u32(&s_empty[slot]), (unsigned int)(it / QS_SLOTS - 1) & 1u, p.err);
+                    mbar_wait(smem_u32(&s_empty[slot]), (unsigned int)(it / nslots - 1) & 1u, p.err);
                 }
                 const unsigned int bar = smem_u32(&s_full[slot]);
                 mbar_expect_tx(bar, (unsigned int)len * 16u);
@@ -238,9 +287,133 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
     pdl_wait();                    // partials, counters and outputs may still be in use by the kernel ahead
     const int K = p.K;
     const unsigned int ninf = BF16 ? 0xff80ff80u : 0xff800000u;
-    const unsigned int floor2 = 0xf149f149u;     // bf16 pair of -1e30: keeps 0 * x finite for x = -inf
-    int it = 0;
+    int it = 0;                    // items of this share consumed so far (the producer counts the same way)
+    int seg = 0;                   // segments of this share finished so far (parity selects the s_top / s_wstat copy)
     long long g = g0;
+
+    // One item: waits for its slot, keeps the maxima of the thread's QS_VPT vectors in vm[], folds the item into the
+    // thread's running (max, sum e^(x-max), sum x e^(x-max)).
+    auto consume_item = [&](int slot, int v_item, int len, float* vm, float& m_t, float2& s2, float2& u2) {
+        mbar_wait(smem_u32(&s_full[slot]), (unsigned int)(it / nslots) & 1u, p.err);
+        const uint4* st = reinterpret_cast<const uint4*>(slots_gen + (size_t)slot * (QS_ITEM_VECS * 16));
+        uint4 d[QS_VPT];
+        float imax = -CUDART_INF_F;
+#pragma unroll
+        for (int j = 0; j < QS_VPT; ++j) {
+            const int vl = tid + j * QS_CONSUMERS;
+            d[j] = (vl < len) ? st[vl] : make_uint4(ninf, ninf, ninf, ninf);
+            if (v_item + vl == p.nvec - 1 && p.nvec * VE != p.vocab) {      // the row's last vector runs past vocab
+                unsigned int* wd = reinterpret_cast<unsigned int*>(&d[j]);
+#pragma unroll
+                for (int e = 0; e < VE; ++e)
+                    if ((p.nvec - 1) * VE + e >= p.vocab) {
+                        if (BF16) wd[e >> 1] = (e & 1) ? ((wd[e >> 1] & 0x0000ffffu) | 0xff800000u)
+                                                       : ((wd[e >> 1] & 0xffff0000u) | 0x0000ff80u);
+                        else wd[e] = 0xff800000u;
+                    }
+            }
+            if (BF16) {
+                const __nv_bfloat162 a = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&d[j].x),
+                                                *reinterpret_cast<const __nv_bfloat162*>(&d[j].y));
+                const __nv_bfloat162 b = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&d[j].z),
+                                                *reinterpret_cast<const __nv_bfloat162*>(&d[j].w));
+                const __nv_bfloat162 c = __hmax2(a, b);
+                const unsigned int cw = *reinterpret_cast<const unsigned int*>(&c);
+                vm[j] = fmaxf(bf16_lo(cw), bf16_hi(cw));
+            } else {
+                vm[j] = fmaxf(fmaxf(__uint_as_float(d[j].x), __uint_as_float(d[j].y)),
+                              fmaxf(__uint_as_float(d[j].z), __uint_as_float(d[j].w)));
+            }
+            imax = fmaxf(imax, vm[j]);
+        }
+        if (imax > m_t) {                         // the thread's maximum grows: rescale its sums
+            const float f = (m_t == -CUDART_INF_F) ? 0.f : ex2f((m_t - imax) * LOG2E);
+            s2.x *= f; s2.y *= f; u2.x *= f; u2.y *= f;
+            m_t = imax;
+        }
+        const float nml = (m_t == -CUDART_INF_F) ? 0.f : -m_t * LOG2E;
+        const float2 l2 = make_float2(LOG2E, LOG2E), n2 = make_float2(nml, nml);
+        const unsigned int floor2 = 0xf149f149u;  // bf16 pair of -1e30: keeps 0 * x finite for x = -inf
+#pragma unroll
+        for (int j = 0; j < QS_VPT; ++j) {
+            const unsigned int* wd = reinterpret_cast<const unsigned int*>(&d[j]);
+            if (BF16) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const __nv_bfloat162 cl = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&wd[q]),
+                                                     *reinterpret_cast<const __nv_bfloat162*>(&floor2));
+                    const unsigned int cw = *reinterpret_cast<const unsigned int*>(&cl);
+                    const float2 x = make_float2(bf16_lo(cw), bf16_hi(cw));
+                    const float2 t = fma2_ftz(x, l2, n2);
+                    const float2 e = make_float2(ex2f(t.x), ex2f(t.y));
+                    s2 = add2_ftz(s2, e);
+                    u2 = fma2_ftz(e, x, u2);
+                }
+            } else {
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    const float2 x = make_float2(fmaxf(__uint_as_float(wd[2 * q]), -1e30f),
+                                                 fmaxf(__uint_as_float(wd[2 * q + 1]), -1e30f));
+                    const float2 t = fma2_ftz(x, l2, n2);
+                    const float2 e = make_float2(ex2f(t.x), ex2f(t.y));
+                    s2 = add2_ftz(s2, e);
+                    u2 = fma2_ftz(e, x, u2);
+                }
+            }
+        }
+    };
+    // A lower bound of the segment's K-th largest logit.  Maxima of disjoint element sets are distinct elements, so
+    // the K-th largest of any such family is a bound.  With at least one full item behind the segment: the CTA's 32
+    // half-warp maxima (published in shared memory; an entry another warp has not refreshed yet is an older maximum
+    // of the same segment, still an element of it).  Shorter: this warp's own 32 lane maxima.
+    auto kth_bound = [&](float m_t, bool full_item, bool barrier) -> float {
+        float w = m_t;
+        if (full_item) {
+            float hm = m_t;
+            hm = fmaxf(hm, __shfl_xor_sync(HS_FULL_MASK, hm, 1));
+            hm = fmaxf(hm, __shfl_xor_sync(HS_FULL_MASK, hm, 2));
+            hm = fmaxf(hm, __shfl_xor_sync(HS_FULL_MASK, hm, 4));
+            hm = fmaxf(hm, __shfl_xor_sync(HS_FULL_MASK, hm, 8));
+            if ((lane & 15) == 0) s_gm[warp * 2 + (lane >> 4)] = hm;
+            if (barrier) bar_sync(1, QS_CONSUMERS);          // every warp has published maxima of this segment
+            else __syncwarp();
+            w = s_gm[lane];
+        } else if (barrier) {
+            bar_sync(1, QS_CONSUMERS);                       // (the same barrier count for every warp)
+        }
+        int ge = 0;                                          // values >= this lane's: independent shuffles
+#pragma unroll
+        for (int j = 0; j < 32; ++j) ge += (__shfl_sync(HS_FULL_MASK, w, j) >= w);
+        return warp_max(ge >= K ? w : -CUDART_INF_F);
+    };
+    // Candidates of one item: the warp works through the vectors whose maximum reaches the bound, four at a time
+    // (eight lanes per vector, one element each, read back from the item's slot in shared memory).
+    auto scan_item = [&](int slot, int v_item, const float* vm, float tau) {
+        unsigned int hits = 0u;
+#pragma unroll
+        for (int j = 0; j < QS_VPT; ++j) hits |= (vm[j] >= tau && vm[j] > -CUDART_INF_F) ? (1u << j) : 0u;
+        unsigned int any = __ballot_sync(HS_FULL_MASK, hits != 0u);
+        while (any) {
+            const int src = __ffs(any) - 1;
+            unsigned int m = __shfl_sync(HS_FULL_MASK, hits, src);
+            any &= any - 1;                                   // (a lane has at most QS_VPT = 4 hit vectors: one round)
+            for (int q = (lane >> 3); q > 0; --q) m &= m - 1; // lanes 8q .. 8q+7 take the q-th hit vector
+            const int e = lane & 7;
+            if (m && e < VE) {
+                const int j = __ffs(m) - 1;
+                const int vl = (warp * 32 + src) + j * QS_CONSUMERS;
+                const unsigned char* vp = slots_gen + (size_t)slot * (QS_ITEM_VECS * 16) + (size_t)vl * 16;
+                const float x = BF16 ? __uint_as_float((unsigned int)reinterpret_cast<const unsigned short*>(vp)[e] << 16)
+                                     : reinterpret_cast<const float*>(vp)[e];
+                const int idx = (v_item + vl) * VE + e;
+                if (x >= tau && x > -CUDART_INF_F && idx < p.vocab) {
+                    const int sl = atomicAdd(&s_cnt, 1);
+                    if (sl < CAND_CAP) s_list[sl] = make_key(x, idx);
+                }
+            }
+        }
+    };
+
     while (g < g1) {
         // ---- one segment: the part [g, seg_end) of this share inside row `row` ------------------------------------
         const int row = (int)(g / p.nvec);
@@ -248,195 +421,86 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
         const int sv0 = (int)(g - row_g0);
         const int sv1 = (int)(min(g1, row_g0 + p.nvec) - row_g0);
         const char* rowp = (const char*)p.logits + (size_t)row * p.row_stride * esz;
+        unsigned long long* top = s_top[seg & 1];
         float m_t = -CUDART_INF_F;                // running maximum of this thread's logits of the segment
         float2 s2 = make_float2(0.f, 0.f), u2 = make_float2(0.f, 0.f);
-        float tau = -CUDART_INF_F;                // lower bound of the K-th largest logit of the segment
+        float tau;                                // lower bound of the K-th largest logit of the segment
         int v = sv0;
-        bool first_window = true;
-        while (v < sv1) {
-            // ---- a window of up to QS_WINDOW items -------------------------------------------------------------
-            float vmx[QS_WINDOW * QS_VPT];
-            int w_slot[QS_WINDOW], w_v0[QS_WINDOW], w_len[QS_WINDOW];
-            int nitems = 0;
-            float wmax = -CUDART_INF_F;
-            const int win_v0 = v;
+        int items_done = 0;
+        {
+            // ---- first window: up to QS_WINDOW items are held, the bound is taken from all of them -----------------
+            float vmx[QS_WINDOW][QS_VPT];
+            int w_slot[QS_WINDOW], w_v0[QS_WINDOW];
 #pragma unroll
             for (int wi = 0; wi < QS_WINDOW; ++wi) {
-#pragma unroll
-                for (int j = 0; j < QS_VPT; ++j) vmx[wi * QS_VPT + j] = -CUDART_INF_F;
-                w_slot[wi] = 0; w_v0[wi] = 0; w_len[wi] = 0;
+                w_slot[wi] = -1; w_v0[wi] = 0;
                 if (v < sv1) {
                     const int len = min(QS_ITEM_VECS, sv1 - v);
-                    const int slot = it % QS_SLOTS;
-                    w_slot[wi] = slot; w_v0[wi] = v; w_len[wi] = len;
-                    nitems = wi + 1;
-                    mbar_wait(smem_u32(&s_full[slot]), (unsigned int)(it / QS_SLOTS) & 1u, p.err);
-                    const uint4* st = reinterpret_cast<const uint4*>(slots_gen + (size_t)slot * (QS_ITEM_VECS * 16));
-                    uint4 d[QS_VPT];
-                    float imax = -CUDART_INF_F;
-#pragma unroll
-                    for (int j = 0; j < QS_VPT; ++j) {
-                        const int vl = tid + j * QS_CONSUMERS;
-                        d[j] = (vl < len) ? st[vl] : make_uint4(ninf, ninf, ninf, ninf);
-                        if (v + vl == p.nvec - 1 && p.nvec * VE != p.vocab) {      // the row's last vector runs past vocab
-                            unsigned int* wd = reinterpret_cast<unsigned int*>(&d[j]);
-#pragma unroll
-                            for (int e = 0; e < VE; ++e)
-                                if ((p.nvec - 1) * VE + e >= p.vocab) {
-                                    if (BF16) wd[e >> 1] = (e & 1) ? ((wd[e >> 1] & 0x0000ffffu) | 0xff800000u)
-                                                                   : ((wd[e >> 1] & 0xffff0000u) | 0x0000ff80u);
-                                    else wd[e] = 0xff800000u;
-                                }
-                        }
-                        float vm;
-                        if (BF16) {
-                            const __nv_bfloat162 a = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&d[j].x),
-                                                            *reinterpret_cast<const __nv_bfloat162*>(&d[j].y));
-                            const __nv_bfloat162 b = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&d[j].z),
-                                                            *reinterpret_cast<const __nv_bfloat162*>(&d[j].w));
-                            const __nv_bfloat162 c = __hmax2(a, b);
-                            const unsigned int cw = *reinterpret_cast<const unsigned int*>(&c);
-                            vm = fmaxf(bf16_lo(cw), bf16_hi(cw));
-                        } else {
-                            vm = fmaxf(fmaxf(__uint_as_float(d[j].x), __uint_as_float(d[j].y)),
-                                       fmaxf(__uint_as_float(d[j].z), __uint_as_float(d[j].w)));
-                        }
-                        vmx[wi * QS_VPT + j] = vm;
-                        imax = fmaxf(imax, vm);
-                    }
-                    if (imax > m_t) {                         // the thread's maximum grows: rescale its sums
-                        const float f = (m_t == -CUDART_INF_F) ? 0.f : ex2f((m_t - imax) * LOG2E);
-                        s2.x *= f; s2.y *= f; u2.x *= f; u2.y *= f;
-                        m_t = imax;
-                    }
-                    wmax = fmaxf(wmax, imax);
-                    const float nml = (m_t == -CUDART_INF_F) ? 0.f : -m_t * LOG2E;
-                    const float2 l2 = make_float2(LOG2E, LOG2E), n2 = make_float2(nml, nml);
-#pragma unroll
-                    for (int j = 0; j < QS_VPT; ++j) {
-                        if (BF16) {
-                            const unsigned int* wd = reinterpret_cast<const unsigned int*>(&d[j]);
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                const __nv_bfloat162 cl = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&wd[q]),
-                                                                 *reinterpret_cast<const __nv_bfloat162*>(&floor2));
-                                const unsigned int cw = *reinterpret_cast<const unsigned int*>(&cl);
-                                const float2 x = make_float2(bf16_lo(cw), bf16_hi(cw));
-                                const float2 t = fma2_ftz(x, l2, n2);
-                                const float2 e = make_float2(ex2f(t.x), ex2f(t.y));
-                                s2 = add2_ftz(s2, e);
-                                u2 = fma2_ftz(e, x, u2);
-                            }
-                        } else {
-                            const unsigned int* wd = reinterpret_cast<const unsigned int*>(&d[j]);
-#pragma unroll
-                            for (int q = 0; q < 2; ++q) {
-                                const float2 x = make_float2(fmaxf(__uint_as_float(wd[2 * q]), -1e30f),
-                                                             fmaxf(__uint_as_float(wd[2 * q + 1]), -1e30f));
-                                const float2 t = fma2_ftz(x, l2, n2);
-                                const float2 e = make_float2(ex2f(t.x), ex2f(t.y));
-                                s2 = add2_ftz(s2, e);
-                                u2 = fma2_ftz(e, x, u2);
-                            }
-                        }
-                    }
-                    v += len;
-                    ++it;
+                    w_slot[wi] = it % nslots; w_v0[wi] = v;
+                    consume_item(w_slot[wi], v, len, vmx[wi], m_t, s2, u2);
+                    v += len; ++it; ++items_done;
                 }
             }
-            // ---- a lower bound of the segment's K-th largest logit -------------------------------------------
-            // Maxima of disjoint element sets are distinct elements, so the K-th largest of any such family is a
-            // bound.  A window of at least one full item: the CTA's 32 half-warp maxima (published in shared memory;
-            // an entry another warp has not refreshed yet is an older maximum of the same segment, still an element
-            // of it).  Shorter: this warp's own 32 lane maxima.
-            const int win_vecs = v - win_v0;
-            if (win_vecs >= QS_ITEM_VECS) {
-                float hm = m_t;
-                hm = fmaxf(hm, __shfl_xor_sync(HS_FULL_MASK, hm, 1));
-                hm = fmaxf(hm, __shfl_xor_sync(HS_FULL_MASK, hm, 2));
-                hm = fmaxf(hm, __shfl_xor_sync(HS_FULL_MASK, hm, 4));
-                hm = fmaxf(hm, __shfl_xor_sync(HS_FULL_MASK, hm, 8));
-                if ((lane & 15) == 0) s_gm[warp * 2 + (lane >> 4)] = hm;
-                if (first_window) bar_sync(1, QS_CONSUMERS);      // every warp has published maxima of this segment
-                else __syncwarp();
-                tau = fmaxf(tau, warp_kth_largest(s_gm[lane], K, lane));
-            } else {
-                if (first_window) bar_sync(1, QS_CONSUMERS);      // (keeps the barrier count the same for every warp)
-                tau = fmaxf(tau, warp_kth_largest(m_t, K, lane));
-            }
-            first_window = false;
-            // ---- candidates: lanes whose window maximum reaches the bound re-scan their vectors ------------------
-            if (wmax >= tau && wmax > -CUDART_INF_F) {
-#pragma unroll 1
-                for (int i = 0; i < nitems * QS_VPT; ++i) {
-                    float vm = -CUDART_INF_F;
+            tau = kth_bound(m_t, v - sv0 >= QS_ITEM_VECS, true);
 #pragma unroll
-                    for (int q = 0; q < QS_WINDOW * QS_VPT; ++q) vm = (q == i) ? vmx[q] : vm;
-                    if (vm >= tau && vm > -CUDART_INF_F) {
-                        const int wi = i / QS_VPT, j = i - wi * QS_VPT;
-                        int slot = 0, iv0 = 0;
-#pragma unroll
-                        for (int q = 0; q < QS_WINDOW; ++q) { slot = (q == wi) ? w_slot[q] : slot; iv0 = (q == wi) ? w_v0[q] : iv0; }
-                        const int vl = tid + j * QS_CONSUMERS;
-                        const uint4 dv = reinterpret_cast<const uint4*>(slots_gen + (size_t)slot * (QS_ITEM_VECS * 16))[vl];
-                        float x[8];
-                        unpack<BF16>(dv, x);
-                        const int base = (iv0 + vl) * VE;
-#pragma unroll
-                        for (int e = 0; e < VE; ++e) {
-                            if (x[e] >= tau && x[e] > -CUDART_INF_F && base + e < p.vocab) {
-                                const int sl = atomicAdd(&s_cnt, 1);
-                                if (sl < CAND_CAP) s_list[sl] = make_key(x[e], base + e);
-                            }
-                        }
-                    }
-                }
-            }
-            // ---- the window's slots go back to the producer -------------------------------------------------------
+            for (int wi = 0; wi < QS_WINDOW; ++wi)
+                if (w_slot[wi] >= 0) scan_item(w_slot[wi], w_v0[wi], vmx[wi], tau);
             __syncwarp();
-            if (lane == 0)
-                for (int wi = 0; wi < nitems; ++wi) {
-                    int slot = 0;
+            if (lane == 0) {
 #pragma unroll
-                    for (int q = 0; q < QS_WINDOW; ++q) slot = (q == wi) ? w_slot[q] : slot;
-                    mbar_arrive(smem_u32(&s_empty[slot]));
-                }
+                for (int wi = 0; wi < QS_WINDOW; ++wi)
+                    if (w_slot[wi] >= 0) mbar_arrive(smem_u32(&s_empty[w_slot[wi]]));
+            }
+        }
+        // ---- the rest of the segment item by item: scanned against the bound and handed back at once; the bound is
+        // refreshed whenever the number of items read reaches a power of two -----------------------------------------
+        while (v < sv1) {
+            float vm[QS_VPT];
+            const int len = min(QS_ITEM_VECS, sv1 - v);
+            const int slot = it % nslots;
+            consume_item(slot, v, len, vm, m_t, s2, u2);
+            ++items_done;
+            if ((items_done & (items_done - 1)) == 0) tau = fmaxf(tau, kth_bound(m_t, true, false));
+            scan_item(slot, v, vm, tau);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));
+            v += len; ++it;
         }
         // ---- end of the segment: warp, then CTA reduction of (max, s, u); Top-K of the candidates ------------------
         {
             const float wm = warp_max(m_t);
             const float f = (m_t == -CUDART_INF_F) ? 0.f : ex2f((m_t - wm) * LOG2E);
             const float ws = warp_sum((s2.x + s2.y) * f), wu = warp_sum((u2.x + u2.y) * f);
-            if (lane == 0) { s_wstat[warp][0] = wm; s_wstat[warp][1] = ws; s_wstat[warp][2] = wu; }
+            if (lane == 0) { s_wstat[seg & 1][warp][0] = wm; s_wstat[seg & 1][warp][1] = ws; s_wstat[seg & 1][warp][2] = wu; }
         }
+        if (tid < HS_MAX_TOPK) top[tid] = 0ull;       // (this copy was last read two segments ago)
         bar_sync(1, QS_CONSUMERS);                    // all candidates are pushed, all warp sums written
         const int ncand = s_cnt;
-        if (ncand <= CAND_CAP) rank_select(s_list, ncand, K, s_top, tid, QS_CONSUMERS);
-        else topk_by_rounds<BF16>(rowp, sv0, sv1, p.vocab, K, s_top, s_red, tid, QS_CONSUMERS, 1);   // heavy ties
-        bar_sync(1, QS_CONSUMERS);                    // s_top is complete
-        // segments of this row: shares c_first .. c_last
-        const int c_first = (int)(row_g0 / p.per), c_last = (int)((row_g0 + p.nvec - 1) / p.per);
-        const int nseg = c_last - c_first + 1;
+        if (ncand <= CAND_CAP) rank_select(s_list, ncand, K, top, tid, QS_CONSUMERS);
+        else topk_by_rounds<BF16>(rowp, sv0, sv1, p.vocab, K, top, s_red, tid, QS_CONSUMERS, 1);   // heavy ties
+        bar_sync(1, QS_CONSUMERS);                    // the Top-K is complete; s_list and s_cnt are free again
+        int c_first, nseg;
+        shares_of_row(p, row, c_first, nseg);
         if (warp == 0) {
+            if (lane == 0) s_cnt = 0;                 // (the next push comes after the next segment's first barrier)
             // the sixteen warps' (max, s, u) in a fixed order
-            const float wm = lane < QS_CONSUMERS / 32 ? s_wstat[lane & 15][0] : -CUDART_INF_F;
+            const float wm = lane < NW ? s_wstat[seg & 1][lane & (NW - 1)][0] : -CUDART_INF_F;
             const float M = warp_max(wm);
-            const float f = (lane >= QS_CONSUMERS / 32 || wm == -CUDART_INF_F) ? 0.f : ex2f((wm - M) * LOG2E);
-            const float S = s_wstat[lane & 15][1] * f, U = s_wstat[lane & 15][2] * f;
+            const float f = (lane >= NW || wm == -CUDART_INF_F) ? 0.f : ex2f((wm - M) * LOG2E);
+            const float S = s_wstat[seg & 1][lane & (NW - 1)][1] * f, U = s_wstat[seg & 1][lane & (NW - 1)][2] * f;
             float St = 0.f, Ut = 0.f;
 #pragma unroll
-            for (int w = 0; w < QS_CONSUMERS / 32; ++w) {
+            for (int w = 0; w < NW; ++w) {
                 St += __shfl_sync(HS_FULL_MASK, S, w);
                 Ut += __shfl_sync(HS_FULL_MASK, U, w);
             }
             if (nseg == 1) {
-                finalize_row(p, row, M, St, Ut, s_top, lane);
-                if (lane == 0) { s_flag = 0; s_cnt = 0; }
+                // the whole row lay in this share: the other warps are already on their way to the next segment
+                finalize_row(p, row, M, St, Ut, top, lane);
             } else {
-                // partial slot: two per share, the leading one for a row that began in an earlier share
-                const int ps = 2 * blockIdx.x + (row_g0 < g0 ? 0 : 1);
+                const int ps = partial_slot(p, row, blockIdx.x);
                 if (lane == 0) p.part_stats[ps] = make_float4(M, St, Ut, 0.f);
-                if (lane < HS_MAX_TOPK) p.part_keys[(size_t)ps * HS_MAX_TOPK + lane] = (lane < K) ? s_top[lane] : 0ull;
+                if (lane < HS_MAX_TOPK) p.part_keys[(size_t)ps * HS_MAX_TOPK + lane] = (lane < K) ? top[lane] : 0ull;
                 __syncwarp();
                 if (lane == 0) {
                     __threadfence();
@@ -444,38 +508,35 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
                     if (last) p.row_cnt[row] = 0;              // ready for the next launch
                     __threadfence();
                     s_flag = last;
-                    s_cnt = 0;
                 }
             }
         }
-        bar_sync(1, QS_CONSUMERS);                    // s_flag; s_top and s_list may be reused
-        if (s_flag) {
-            // ---- the last share of a split row merges the row's partials -------------------------------------------
-            if (tid < HS_MAX_TOPK) s_top[tid] = 0ull;
-            for (int t = tid; t < nseg * HS_MAX_TOPK; t += QS_CONSUMERS) {
-                const int c = c_first + t / HS_MAX_TOPK;
-                const int ps = 2 * c + (row_g0 < (long long)c * p.per ? 0 : 1);
-                s_list[t] = __ldcg(&p.part_keys[(size_t)ps * HS_MAX_TOPK + (t % HS_MAX_TOPK)]);
-            }
-            bar_sync(1, QS_CONSUMERS);
-            rank_select(s_list, nseg * HS_MAX_TOPK, K, s_top, tid, QS_CONSUMERS);
-            bar_sync(1, QS_CONSUMERS);
-            if (warp == 0) {
-                float m = -CUDART_INF_F, cs = 0.f, cu = 0.f;
-                if (lane < nseg) {
-                    const int c = c_first + lane;
-                    const int ps = 2 * c + (row_g0 < (long long)c * p.per ? 0 : 1);
-                    const float4 stv = __ldcg(&p.part_stats[ps]);
-                    m = stv.x; cs = stv.y; cu = stv.z;
+        if (nseg > 1) {
+            bar_sync(1, QS_CONSUMERS);                // s_flag
+            if (s_flag) {
+                // ---- the last share of a split row merges the row's partials ---------------------------------------
+                if (tid < HS_MAX_TOPK) top[tid] = 0ull;
+                for (int t = tid; t < nseg * HS_MAX_TOPK; t += QS_CONSUMERS) {
+                    const int ps = partial_slot(p, row, c_first + t / HS_MAX_TOPK);
+                    s_list[t] = __ldcg(&p.part_keys[(size_t)ps * HS_MAX_TOPK + (t % HS_MAX_TOPK)]);
                 }
-                const float M = warp_max(m);
-                const float f = (m == -CUDART_INF_F) ? 0.f : ex2f((m - M) * LOG2E);
-                const float S = warp_sum(cs * f), U = warp_sum(cu * f);
-                finalize_row(p, row, M, S, U, s_top, lane);
+                bar_sync(1, QS_CONSUMERS);
+                rank_select(s_list, nseg * HS_MAX_TOPK, K, top, tid, QS_CONSUMERS);
+                bar_sync(1, QS_CONSUMERS);
+                if (warp == 0) {
+                    float m = -CUDART_INF_F, cs = 0.f, cu = 0.f;
+                    if (lane < nseg) {
+                        const float4 stv = __ldcg(&p.part_stats[partial_slot(p, row, c_first + lane)]);
+                        m = stv.x; cs = stv.y; cu = stv.z;
+                    }
+                    const float M = warp_max(m);
+                    const float f = (m == -CUDART_INF_F) ? 0.f : ex2f((m - M) * LOG2E);
+                    const float S = warp_sum(cs * f), U = warp_sum(cu * f);
+                    finalize_row(p, row, M, S, U, top, lane);
+                }
             }
-            bar_sync(1, QS_CONSUMERS);
         }
-        if (tid < HS_MAX_TOPK) s_top[tid] = 0ull;     // (next written after the next segment's first barrier)
+        ++seg;
         g = row_g0 + sv1;
     }
 }
@@ -576,6 +637,9 @@ static void fill_common(QuantParams& p, const hs_tree_batch* tree, const void* l
     p.chunks = 0;
     p.chunk_vecs = 0;
     p.per = 0;
+    p.split = 0;
+    p.extra = 0;
+    p.nslots = QS_SLOTS;
     p.rows = tree->n_nodes_total;
     p.batch = tree->batch;
     p.node_off = tree->node_off;
@@ -592,14 +656,41 @@ static void fill_common(QuantParams& p, const hs_tree_batch* tree, const void* l
     p.err = nullptr;
 }
 
-// Shares of the stream: at most one per SM, at least 32 KiB each, and so large that no row is split over more
-// than QS_MAX_SEGS of them.
-static int quantify_share_vecs(long long total_vecs, int nvec, int sm_count) {
-    long long per = (total_vecs + sm_count - 1) / sm_count;
-    const long long floor_row = (nvec + (QS_MAX_SEGS - 2) - 1) / (QS_MAX_SEGS - 2);
-    if (per < floor_row) per = floor_row;
-    if (per < QS_ITEM_VECS) per = QS_ITEM_VECS;
-    return (int)per;
+// Geometry of a launch, one CTA per SM.  With at most one row per SM and rows short enough for the item slots,
+// every SM gets one part of one row (the first rows are cut into one part more than the others so that every SM
+// has work): a CTA then has a single row segment.  With two or more rows per SM every CTA takes whole rows (no row
+// needs a merge).  In between every CTA takes an equal share of the stream, at least one item long and so large
+// that no row is split over more than QS_MAX_SEGS shares.
+static void quantify_geometry(int rows, int nvec, int sm_count, QuantParams& p, int& nctas, size_t& smem) {
+    int S = rows <= sm_count ? sm_count / rows : 0;
+    while (S > 1 && (S + 1 > QS_MAX_SEGS || nvec / (S + 1) < 256)) --S;      // parts of at least 4 KiB
+    const int extra = (S >= 1 && S + 1 <= QS_MAX_SEGS && nvec / (S + 1) >= 256) ? min(rows, sm_count - rows * S) : 0;
+    const int pv_max = S >= 1 ? (nvec + S - 1) / S : 0;
+    if (rows >= 2 * sm_count) {
+        p.split = -1;
+        p.extra = sm_count;
+        p.per = 0;
+        p.nslots = QS_SLOTS;
+        nctas = sm_count;
+    } else if (S >= 1 && pv_max <= QS_SLOTS * QS_ITEM_VECS) {
+        p.split = S;
+        p.extra = extra;
+        p.per = pv_max;
+        p.nslots = (pv_max + QS_ITEM_VECS - 1) / QS_ITEM_VECS;
+        nctas = rows * S + extra;
+    } else {
+        const long long total = (long long)rows * nvec;
+        long long per = (total + sm_count - 1) / sm_count;
+        const long long floor_row = (nvec + (QS_MAX_SEGS - 2) - 1) / (QS_MAX_SEGS - 2);
+        if (per < floor_row) per = floor_row;
+        if (per < QS_ITEM_VECS) per = QS_ITEM_VECS;
+        p.split = 0;
+        p.extra = 0;
+        p.per = (int)per;
+        p.nslots = QS_SLOTS;
+        nctas = (int)((total + per - 1) / per);
+    }
+    smem = (size_t)p.nslots * QS_ITEM_VECS * 16 + 128;
 }
 
 hs_status hs_launch_quantify(hs_ctx* ctx, const hs_tree_batch* tree, const void* logits, hs_dtype dtype,
@@ -608,11 +699,12 @@ hs_status hs_launch_quantify(hs_ctx* ctx, const hs_tree_batch* tree, const void*
     QuantParams p;
     fill_common(p, tree, logits, dtype, row_stride, vocab, policy, out);
     if (p.nvec > QS_ITEM_VECS * 64) return HS_ERR_SHAPE;            // vocabulary beyond 2^20 bf16 / 2^19 fp32 logits
-    const long long total = (long long)p.rows * p.nvec;
-    p.per = quantify_share_vecs(total, p.nvec, ctx->sm_count);
-    const int nctas = (int)((total + p.per - 1) / p.per);
-    const size_t stats_bytes = hs_align_up((size_t)2 * nctas * sizeof(float4), 256);
-    const size_t keys_bytes = (size_t)2 * nctas * HS_MAX_TOPK * sizeof(unsigned long long);
+    int nctas = 0;
+    size_t smem = 0;
+    quantify_geometry(p.rows, p.nvec, ctx->sm_count, p, nctas, smem);
+    const int nparts = p.split ? nctas : 2 * nctas;      // (whole rows: none is used)
+    const size_t stats_bytes = hs_align_up((size_t)nparts * sizeof(float4), 256);
+    const size_t keys_bytes = (size_t)nparts * HS_MAX_TOPK * sizeof(unsigned long long);
     if (stats_bytes + keys_bytes > ctx->scratch_bytes) return HS_ERR_WORKSPACE;
     p.part_stats = (float4*)ctx->scratch;
     p.part_keys = (unsigned long long*)(ctx->scratch + stats_bytes);
@@ -626,8 +718,8 @@ hs_status hs_launch_quantify(hs_ctx* ctx, const hs_tree_batch* tree, const void*
         ctx->quant_ready = true;
     }
     cudaError_t e = dtype == HS_BF16
-        ? hs_launch(quantify_stream_kernel<true>, dim3(nctas), dim3(QS_THREADS), QS_SMEM_BYTES, stream, ctx->pdl, dim3(1, 1, 1), p)
-        : hs_launch(quantify_stream_kernel<false>, dim3(nctas), dim3(QS_THREADS), QS_SMEM_BYTES, stream, ctx->pdl, dim3(1, 1, 1), p);
+        ? hs_launch(quantify_stream_kernel<true>, dim3(nctas), dim3(QS_THREADS), smem, stream, ctx->pdl, dim3(1, 1, 1), p)
+        : hs_launch(quantify_stream_kernel<false>, dim3(nctas), dim3(QS_THREADS), smem, stream, ctx->pdl, dim3(1, 1, 1), p);
     if (e != cudaSuccess) return HS_ERR_CUDA;
     e = hs_launch(tree_scores_kernel, dim3(p.batch), dim3(HS_MAX_NODES), 0, stream, ctx->pdl, dim3(1, 1, 1), p);
     return e == cudaSuccess ? HS_OK : HS_ERR_CUDA;
