@@ -90,7 +90,7 @@ hs_status hs_destroy(hs_ctx* ctx);
  * not written by the immediately preceding kernel of the stream: typically true for the KV cache
  * prefix (appended a step earlier), true for logits only if something else separates producer and
  * call.  Default 0: nothing is read early. */
-#define HS_PREFETCH_LOGITS 1   /* draft logits of hs_entropy_quantify */
+#define HS_PREFETCH_LOGITS 1   /* draft logits and tree arrays (parent, token, node_off) of hs_entropy_quantify */
 #define HS_PREFETCH_KV 2       /* k_cache / v_cache of hs_tree_verify_attention */
 hs_status hs_set_prefetch(hs_ctx* ctx, int32_t flags);
 

@@ -90,6 +90,21 @@ __device__ __forceinline__ void rank_select(const unsigned long long* s_cand, in
     }
 }
 
+// The same by whole warps: warp w takes candidates w, w + nwarp, ...; the 32 lanes compare 32 others at a time.
+__device__ __forceinline__ void rank_select_warps(const unsigned long long* s_cand, int n, int K,
+                                                  unsigned long long* s_top, int warp, int lane, int nwarp) {
+    for (int c = warp; c < n; c += nwarp) {
+        const unsigned long long k = s_cand[c];
+        if (k == 0ull) continue;
+        int rank = 0;
+        for (int j0 = 0; j0 < n && rank < K; j0 += 32) {
+            const int j = j0 + lane;
+            rank += __popc(__ballot_sync(HS_FULL_MASK, j < n && s_cand[j] > k));
+        }
+        if (rank < K && lane == 0) s_top[rank] = k;
+    }
+}
+
 // barrier over the first `nthr` threads of the CTA (a multiple of 32); id 0 is __syncthreads' own
 __device__ __forceinline__ void bar_sync(int id, int nthr) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthr) : "memory");
@@ -232,7 +247,8 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
     __shared__ unsigned long long s_list[CAND_CAP];
     __shared__ unsigned long long s_top[2][HS_MAX_TOPK];   // (two copies: a finished row is written out by warp 0
     __shared__ unsigned long long s_red[NW];               //  while the other warps read the next one)
-    __shared__ float s_gm[32];
+    __shared__ __align__(16) float s_gm[32];
+    __shared__ __align__(16) float s_lm[NW][32];
     __shared__ float s_wstat[2][NW][3];
     __shared__ int s_cnt;
     __shared__ int s_flag;
@@ -260,17 +276,17 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
         // ---- producer: one lane walks the share item by item ----------------------------------------------------
         if (lane == 0) {
             long long g = g0;
-            int it = 0;
+            int it = 0, slot = 0;
+            unsigned int epar = 1u;          // parity of the slot's `empty` barrier before its first completion
             bool waited = false;
             if (!p.prefetch) { pdl_wait(); waited = true; }
             while (g < g1) {
                 const int row = (int)(g / p.nvec);
                 const int v = (int)(g - (long long)row * p.nvec);
                 const int len = (int)min((long long)min(QS_ITEM_VECS, p.nvec - v), g1 - g);
-                const int slot = it % nslots;
                 if (it >= nslots) {
                     if (!waited) { pdl_wait(); waited = true; }     // (nothing of this kernel is written by the producer)
-                    mbar_wait(smem_u32(&s_empty[slot]), (unsigned int)(it / nslots - 1) & 1u, p.err);
+                    mbar_wait(smem_u32(&s_empty[slot]), epar, p.err);
                 }
                 const unsigned int bar = smem_u32(&s_full[slot]);
                 mbar_expect_tx(bar, (unsigned int)len * 16u);
@@ -278,6 +294,7 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
                           (const char*)p.logits + (size_t)row * p.row_stride * esz + (size_t)v * 16, (unsigned int)len * 16u, bar);
                 g += len;
                 ++it;
+                if (++slot == nslots) { slot = 0; epar ^= 1u; }
             }
         }
         return;
@@ -287,31 +304,46 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
     pdl_wait();                    // partials, counters and outputs may still be in use by the kernel ahead
     const int K = p.K;
     const unsigned int ninf = BF16 ? 0xff80ff80u : 0xff800000u;
-    int it = 0;                    // items of this share consumed so far (the producer counts the same way)
+    int cslot = 0;                 // slot of the next item and the parity of its `full` barrier (the producer fills
+    unsigned int cpar = 0u;        // the slots round-robin in the same order)
     int seg = 0;                   // segments of this share finished so far (parity selects the s_top / s_wstat copy)
     long long g = g0;
 
     // One item: waits for its slot, keeps the maxima of the thread's QS_VPT vectors in vm[], folds the item into the
     // thread's running (max, sum e^(x-max), sum x e^(x-max)).
     auto consume_item = [&](int slot, int v_item, int len, float* vm, float& m_t, float2& s2, float2& u2) {
-        mbar_wait(smem_u32(&s_full[slot]), (unsigned int)(it / nslots) & 1u, p.err);
+        mbar_wait(smem_u32(&s_full[slot]), cpar, p.err);
+        if (++cslot == nslots) { cslot = 0; cpar ^= 1u; }
         const uint4* st = reinterpret_cast<const uint4*>(slots_gen + (size_t)slot * (QS_ITEM_VECS * 16));
         uint4 d[QS_VPT];
         float imax = -CUDART_INF_F;
+        if (len == QS_ITEM_VECS) {                                           // (the usual case: no lane is idle)
+#pragma unroll
+            for (int j = 0; j < QS_VPT; ++j) d[j] = st[tid + j * QS_CONSUMERS];
+        } else {
+#pragma unroll
+            for (int j = 0; j < QS_VPT; ++j) {
+                const int vl = tid + j * QS_CONSUMERS;
+                d[j] = (vl < len) ? st[vl] : make_uint4(ninf, ninf, ninf, ninf);
+            }
+        }
+        if (v_item + len == p.nvec && p.nvec * VE != p.vocab) {               // the row's last vector runs past vocab
+#pragma unroll
+            for (int j = 0; j < QS_VPT; ++j) {
+                if (v_item + tid + j * QS_CONSUMERS == p.nvec - 1) {
+                    unsigned int* wd = reinterpret_cast<unsigned int*>(&d[j]);
+#pragma unroll
+                    for (int e = 0; e < VE; ++e)
+                        if ((p.nvec - 1) * VE + e >= p.vocab) {
+                            if (BF16) wd[e >> 1] = (e & 1) ? ((wd[e >> 1] & 0x0000ffffu) | 0xff800000u)
+                                                           : ((wd[e >> 1] & 0xffff0000u) | 0x0000ff80u);
+                            else wd[e] = 0xff800000u;
+                        }
+                }
+            }
+        }
 #pragma unroll
         for (int j = 0; j < QS_VPT; ++j) {
-            const int vl = tid + j * QS_CONSUMERS;
-            d[j] = (vl < len) ? st[vl] : make_uint4(ninf, ninf, ninf, ninf);
-            if (v_item + vl == p.nvec - 1 && p.nvec * VE != p.vocab) {      // the row's last vector runs past vocab
-                unsigned int* wd = reinterpret_cast<unsigned int*>(&d[j]);
-#pragma unroll
-                for (int e = 0; e < VE; ++e)
-                    if ((p.nvec - 1) * VE + e >= p.vocab) {
-                        if (BF16) wd[e >> 1] = (e & 1) ? ((wd[e >> 1] & 0x0000ffffu) | 0xff800000u)
-                                                       : ((wd[e >> 1] & 0xffff0000u) | 0x0000ff80u);
-                        else wd[e] = 0xff800000u;
-                    }
-            }
             if (BF16) {
                 const __nv_bfloat162 a = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&d[j].x),
                                                 *reinterpret_cast<const __nv_bfloat162*>(&d[j].y));
@@ -367,7 +399,7 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
     // half-warp maxima (published in shared memory; an entry another warp has not refreshed yet is an older maximum
     // of the same segment, still an element of it).  Shorter: this warp's own 32 lane maxima.
     auto kth_bound = [&](float m_t, bool full_item, bool barrier) -> float {
-        float w = m_t;
+        const float4* fam;                                   // the family of 32 maxima, read back as eight float4
         if (full_item) {
             float hm = m_t;
             hm = fmaxf(hm, __shfl_xor_sync(HS_FULL_MASK, hm, 1));
@@ -377,13 +409,20 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
             if ((lane & 15) == 0) s_gm[warp * 2 + (lane >> 4)] = hm;
             if (barrier) bar_sync(1, QS_CONSUMERS);          // every warp has published maxima of this segment
             else __syncwarp();
-            w = s_gm[lane];
-        } else if (barrier) {
-            bar_sync(1, QS_CONSUMERS);                       // (the same barrier count for every warp)
+            fam = reinterpret_cast<const float4*>(s_gm);
+        } else {
+            s_lm[warp][lane] = m_t;
+            if (barrier) bar_sync(1, QS_CONSUMERS);          // (the same barrier count for every warp)
+            else __syncwarp();
+            fam = reinterpret_cast<const float4*>(s_lm[warp]);
         }
-        int ge = 0;                                          // values >= this lane's: independent shuffles
+        const float w = reinterpret_cast<const float*>(fam)[lane];
+        int ge = 0;                                          // members >= this lane's
 #pragma unroll
-        for (int j = 0; j < 32; ++j) ge += (__shfl_sync(HS_FULL_MASK, w, j) >= w);
+        for (int j = 0; j < 8; ++j) {
+            const float4 f4 = fam[j];
+            ge += (f4.x >= w) + (f4.y >= w) + (f4.z >= w) + (f4.w >= w);
+        }
         return warp_max(ge >= K ? w : -CUDART_INF_F);
     };
     // Candidates of one item: the warp works through the vectors whose maximum reaches the bound, four at a time
@@ -436,9 +475,9 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
                 w_slot[wi] = -1; w_v0[wi] = 0;
                 if (v < sv1) {
                     const int len = min(QS_ITEM_VECS, sv1 - v);
-                    w_slot[wi] = it % nslots; w_v0[wi] = v;
+                    w_slot[wi] = cslot; w_v0[wi] = v;
                     consume_item(w_slot[wi], v, len, vmx[wi], m_t, s2, u2);
-                    v += len; ++it; ++items_done;
+                    v += len; ++items_done;
                 }
             }
             tau = kth_bound(m_t, v - sv0 >= QS_ITEM_VECS, true);
@@ -457,14 +496,14 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
         while (v < sv1) {
             float vm[QS_VPT];
             const int len = min(QS_ITEM_VECS, sv1 - v);
-            const int slot = it % nslots;
+            const int slot = cslot;
             consume_item(slot, v, len, vm, m_t, s2, u2);
             ++items_done;
             if ((items_done & (items_done - 1)) == 0) tau = fmaxf(tau, kth_bound(m_t, true, false));
             scan_item(slot, v, vm, tau);
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));
-            v += len; ++it;
+            v += len;
         }
         // ---- end of the segment: warp, then CTA reduction of (max, s, u); Top-K of the candidates ------------------
         {
@@ -476,18 +515,18 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
         if (tid < HS_MAX_TOPK) top[tid] = 0ull;       // (this copy was last read two segments ago)
         bar_sync(1, QS_CONSUMERS);                    // all candidates are pushed, all warp sums written
         const int ncand = s_cnt;
-        if (ncand <= CAND_CAP) rank_select(s_list, ncand, K, top, tid, QS_CONSUMERS);
+        if (ncand <= CAND_CAP) rank_select_warps(s_list, ncand, K, top, warp, lane, NW);
         else topk_by_rounds<BF16>(rowp, sv0, sv1, p.vocab, K, top, s_red, tid, QS_CONSUMERS, 1);   // heavy ties
         bar_sync(1, QS_CONSUMERS);                    // the Top-K is complete; s_list and s_cnt are free again
         int c_first, nseg;
         shares_of_row(p, row, c_first, nseg);
         if (warp == 0) {
             if (lane == 0) s_cnt = 0;                 // (the next push comes after the next segment's first barrier)
-            // the sixteen warps' (max, s, u) in a fixed order
-            const float wm = lane < NW ? s_wstat[seg & 1][lane & (NW - 1)][0] : -CUDART_INF_F;
+            // the consumer warps' (max, s, u) in a fixed order
+            const float wm = lane < NW ? s_wstat[seg & 1][lane][0] : -CUDART_INF_F;
             const float M = warp_max(wm);
             const float f = (lane >= NW || wm == -CUDART_INF_F) ? 0.f : ex2f((wm - M) * LOG2E);
-            const float S = s_wstat[seg & 1][lane & (NW - 1)][1] * f, U = s_wstat[seg & 1][lane & (NW - 1)][2] * f;
+            const float S = lane < NW ? s_wstat[seg & 1][lane][1] * f : 0.f, U = lane < NW ? s_wstat[seg & 1][lane][2] * f : 0.f;
             float St = 0.f, Ut = 0.f;
 #pragma unroll
             for (int w = 0; w < NW; ++w) {
@@ -505,8 +544,7 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
                 if (lane == 0) {
                     __threadfence();
                     const int last = atomicAdd(&p.row_cnt[row], 1) == nseg - 1;
-                    if (last) p.row_cnt[row] = 0;              // ready for the next launch
-                    __threadfence();
+                    if (last) { p.row_cnt[row] = 0; __threadfence(); }     // (counter ready for the next launch)
                     s_flag = last;
                 }
             }
@@ -516,19 +554,17 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
             if (s_flag) {
                 // ---- the last share of a split row merges the row's partials ---------------------------------------
                 if (tid < HS_MAX_TOPK) top[tid] = 0ull;
+                float4 stv = make_float4(-CUDART_INF_F, 0.f, 0.f, 0.f);       // (warp 0: requested with the keys)
+                if (warp == 0 && lane < nseg) stv = __ldcg(&p.part_stats[partial_slot(p, row, c_first + lane)]);
                 for (int t = tid; t < nseg * HS_MAX_TOPK; t += QS_CONSUMERS) {
                     const int ps = partial_slot(p, row, c_first + t / HS_MAX_TOPK);
                     s_list[t] = __ldcg(&p.part_keys[(size_t)ps * HS_MAX_TOPK + (t % HS_MAX_TOPK)]);
                 }
                 bar_sync(1, QS_CONSUMERS);
-                rank_select(s_list, nseg * HS_MAX_TOPK, K, top, tid, QS_CONSUMERS);
+                rank_select_warps(s_list, nseg * HS_MAX_TOPK, K, top, warp, lane, NW);
                 bar_sync(1, QS_CONSUMERS);
                 if (warp == 0) {
-                    float m = -CUDART_INF_F, cs = 0.f, cu = 0.f;
-                    if (lane < nseg) {
-                        const float4 stv = __ldcg(&p.part_stats[partial_slot(p, row, c_first + lane)]);
-                        m = stv.x; cs = stv.y; cu = stv.z;
-                    }
+                    const float m = stv.x, cs = stv.y, cu = stv.z;
                     const float M = warp_max(m);
                     const float f = (m == -CUDART_INF_F) ? 0.f : ex2f((m - M) * LOG2E);
                     const float S = warp_sum(cs * f), U = warp_sum(cu * f);
@@ -552,7 +588,9 @@ __global__ void __launch_bounds__(HS_MAX_NODES) tree_scores_kernel(const QuantPa
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x;
     pdl_launch_dependents();
-    pdl_wait();                                   // the row statistics come from the kernel ahead
+    // The tree and the logit of every node's token are inputs of the call, not results of the row pass: if the caller
+    // vouches that they were complete before the call (prefetch), they are fetched while the row pass still runs.
+    if (!p.prefetch) pdl_wait();
     const int base = p.node_off[b];
     const int n = p.node_off[b + 1] - base;
     // validation
@@ -564,6 +602,12 @@ __global__ void __launch_bounds__(HS_MAX_NODES) tree_scores_kernel(const QuantPa
         if (tid == 0) bad = (par != -1);
         else bad = (par < 0 || par >= tid || tok < 0 || tok >= p.vocab);
     }
+    float lv = 0.f;
+    if (!bad && tid < n && tid > 0) {
+        const size_t off = (size_t)(base + par) * p.row_stride + tok;
+        lv = p.is_bf16 ? __bfloat162float(((const __nv_bfloat16*)p.logits)[off]) : ((const float*)p.logits)[off];
+    }
+    if (p.prefetch) pdl_wait();                   // the row statistics come from the kernel ahead
     bad = __syncthreads_or(bad);
     if (bad) {
         for (int i = tid; i < n; i += blockDim.x) {
@@ -575,12 +619,7 @@ __global__ void __launch_bounds__(HS_MAX_NODES) tree_scores_kernel(const QuantPa
     }
     if (tid < n) {
         float lc = 0.f;
-        if (tid > 0) {
-            const size_t off = (size_t)(base + par) * p.row_stride + tok;
-            const float lv = p.is_bf16 ? __bfloat162float(((const __nv_bfloat16*)p.logits)[off])
-                                       : ((const float*)p.logits)[off];
-            lc = lv - p.out.row_lse[base + par];
-        }
+        if (tid > 0) lc = lv - p.out.row_lse[base + par];
         s_logc[tid] = lc;
         s_I[tid] = p.entropy_mode == 0 ? p.out.i_topk[base + tid] : p.out.i_trunc[base + tid];
         s_par[tid] = par;
