@@ -26,7 +26,7 @@
 #define ATT_TILE_BYTES (ATT_BN * HS_HEAD_DIM * 2)   // 16 KiB: one K or V tile
 #define ATT_STAGE_BYTES (2 * ATT_TILE_BYTES)
 #define ATT_Q_BYTES (ATT_BM * HS_HEAD_DIM * 2)      // 32 KiB
-#define ATT_PO_STRIDE (HS_HEAD_DIM + 4)             // floats per row of the partial O (padding: bank spread)
+#define ATT_PB_STRIDE (HS_HEAD_DIM * 2 + 16)        // bytes per row of a pushed partial: 128 bf16 of O / l, {max, sum}, padding
 #define LOG2E 1.4426950408889634f
 #define LN2 0.6931471805599453f
 
@@ -90,7 +90,7 @@ __device__ __forceinline__ void prefix_range(int L, int nsplit, int split, int& 
 #define UM_MAP_BYTES 1024                            // output-row map of the rows a CTA merges (<= 65 rows x 8 bytes)
 #define UM_TMEM_COLS 512                             // S of stream g: columns 64 g ..; O: 128 + 128 g ..; P (bf16 pairs): 384 + 32 g ..
 #define UM_STAGES 4
-#define UM_RECV_BYTES (76 * 1024)                    // after the tile loop: partials pushed by the splits of the cluster
+#define UM_RECV_BYTES (40 * 1024)                    // after the tile loop: partials pushed by the splits of the cluster
 #define UM_SMEM_BYTES (UM_STAGES * ATT_STAGE_BYTES + ATT_Q_BYTES + UM_MAP_BYTES + 4096 + 1024)
 
 __global__ void __launch_bounds__(UM_THREADS, 1)
@@ -491,19 +491,23 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
         if (orow >= 0 && p.lse_out && half == 0) p.lse_out[orow] = (mrun + log2f(lrun)) * LN2;
     } else {
         // ---- merge across the splits of the cluster through distributed shared memory ----------------------------
-        // Row rl of the block is merged by CTA owner(rl) = rl * ns / 128.  Every CTA stages its partial
-        // {O row, max, sum} in its own shared memory and one thread PUSHES each owner's rows with a bulk
-        // copy that signals the owner's mbarrier; an owner merges once all ns pieces have landed.
+        // Row rl of the block is merged by CTA owner(rl) = rl * ns / 128.  Every CTA stages its partial of every row,
+        // {O / l as bf16, max, sum}, in its own shared memory and one thread PUSHES each owner's rows with a bulk
+        // copy that signals the owner's mbarrier; an owner merges once all ns pieces have landed: per row the
+        // splits' weights 2^(max_s - max) l_s / sum once, then out = sum_s weight_s (O_s / l_s).  (A normalised
+        // partial is a convex combination of V rows, so bf16 keeps it to 2^-9 of the values' magnitude: the output
+        // is bf16 anyway.)
         const int ns = p.nsplit;
-        // shared memory after the tile loop: [0, 76 KB) partials received from the cluster (others write here,
-        // so only after every CTA of the cluster has left its loop), then this CTA's own staged partial
-        float* po = reinterpret_cast<float*>(smem_gen);                              // [ns][rows_max][ATT_PO_STRIDE]: received
-        float* stage_po = reinterpret_cast<float*>(smem_gen + UM_RECV_BYTES);        // [128][ATT_PO_STRIDE]: own partial
+        // shared memory after the tile loop: [0, UM_RECV_BYTES) partials received from the cluster (others write
+        // here, so only after every CTA of the cluster has left its loop), then this CTA's own staged partial
+        unsigned char* po = smem_gen;                                                // [ns][rows_max] rows of ATT_PB_STRIDE bytes
+        unsigned char* stage_po = smem_gen + UM_RECV_BYTES;                          // [128] rows: own partial
         const unsigned int s_recv = smem_base, s_stage = smem_base + UM_RECV_BYTES;
         const int rows_max = (ATT_BM + ns - 1) / ns + 1;
         const int r_lo = (split * ATT_BM + ns - 1) / ns, r_hi = ((split + 1) * ATT_BM + ns - 1) / ns;   // rows this CTA owns
         long long* s_og = reinterpret_cast<long long*>(gM);               // output row of each owned row (or -1)
-        if (tid == 0) mbar_expect_tx(bar_r, (unsigned int)(ns * (r_hi - r_lo) * ATT_PO_STRIDE * 4));
+        float* s_wt = reinterpret_cast<float*>(gM + UM_MAP_BYTES + 1024);  // [rows owned][ATT_MAX_SPLIT] weights (s_mx / s_lx are done)
+        if (tid == 0) mbar_expect_tx(bar_r, (unsigned int)(ns * (r_hi - r_lo) * ATT_PB_STRIDE));
         if (tid < r_hi - r_lo) {
             const int rg = m0 + r_lo + tid;
             long long og = -1;
@@ -514,17 +518,25 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
             }
             s_og[tid] = og;
         }
+        {
+            const float inv = lrun > 0.f ? 1.f / lrun : 0.f;
 #pragma unroll 1
-        for (int ch = 0; ch < 2 && warp < 8; ++ch) {
-            unsigned int ov[32];
-            load_o(ch, ov);
-            float4* dst = reinterpret_cast<float4*>(stage_po + row * ATT_PO_STRIDE + half * 64 + ch * 32);
+            for (int ch = 0; ch < 2 && warp < 8; ++ch) {
+                unsigned int ov[32];
+                load_o(ch, ov);
+                uint4* dst = reinterpret_cast<uint4*>(stage_po + row * ATT_PB_STRIDE + (half * 64 + ch * 32) * 2);
 #pragma unroll
-            for (int q = 0; q < 8; ++q)
-                dst[q] = make_float4(__uint_as_float(ov[q * 4]), __uint_as_float(ov[q * 4 + 1]),
-                                     __uint_as_float(ov[q * 4 + 2]), __uint_as_float(ov[q * 4 + 3]));
+                for (int q = 0; q < 4; ++q) {
+                    uint4 pk;
+                    pk.x = pack_bf16(__uint_as_float(ov[q * 8 + 0]) * inv, __uint_as_float(ov[q * 8 + 1]) * inv);
+                    pk.y = pack_bf16(__uint_as_float(ov[q * 8 + 2]) * inv, __uint_as_float(ov[q * 8 + 3]) * inv);
+                    pk.z = pack_bf16(__uint_as_float(ov[q * 8 + 4]) * inv, __uint_as_float(ov[q * 8 + 5]) * inv);
+                    pk.w = pack_bf16(__uint_as_float(ov[q * 8 + 6]) * inv, __uint_as_float(ov[q * 8 + 7]) * inv);
+                    dst[q] = pk;
+                }
+            }
+            if (warp < 4) *reinterpret_cast<float2*>(stage_po + row * ATT_PB_STRIDE + HS_HEAD_DIM * 2) = make_float2(mrun, lrun);
         }
-        if (warp < 4) *reinterpret_cast<float2*>(stage_po + row * ATT_PO_STRIDE + HS_HEAD_DIM) = make_float2(mrun, lrun);
         fence_proxy_async_smem();                            // staged rows -> visible to the copy engine
         cluster_arrive();                                    // every CTA of the cluster is done with its tiles:
         cluster_wait();                                      // its stage buffers may now receive partials
@@ -532,48 +544,59 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
             const int o = tid;
             const int o_lo = (o * ATT_BM + ns - 1) / ns, o_hi = ((o + 1) * ATT_BM + ns - 1) / ns;
             if (o_hi > o_lo)
-                bulk_push(cluster_map_addr(s_recv + (unsigned int)(split * rows_max) * ATT_PO_STRIDE * 4, o),
-                          s_stage + (unsigned int)o_lo * ATT_PO_STRIDE * 4, (unsigned int)(o_hi - o_lo) * ATT_PO_STRIDE * 4,
+                bulk_push(cluster_map_addr(s_recv + (unsigned int)(split * rows_max) * ATT_PB_STRIDE, o),
+                          s_stage + (unsigned int)o_lo * ATT_PB_STRIDE, (unsigned int)(o_hi - o_lo) * ATT_PB_STRIDE,
                           cluster_map_addr(bar_r, o));
         }
         mbar_wait(bar_r, 0u, p.err);                         // all ns pieces of this CTA's rows have landed
         cluster_arrive();                                    // (a CTA may leave only when every copy has landed everywhere)
-        // items = (row, float4 column); every item combines one float4 of each split, all from local shared memory
-#pragma unroll 2
-        for (int it = tid; it < (r_hi - r_lo) * 32 && tid < UM_SM_THREADS; it += UM_SM_THREADS) {
-            const int rl = it >> 5, c4 = it & 31;
+        // the splits' weights of every owned row, once
+        if (tid < r_hi - r_lo) {
             float2 ml[ATT_MAX_SPLIT];
-            float4 v[ATT_MAX_SPLIT];
+            float Mx = -CUDART_INF_F;
 #pragma unroll
             for (int s2 = 0; s2 < ATT_MAX_SPLIT; ++s2) {
                 ml[s2] = make_float2(-CUDART_INF_F, 0.f);
-                v[s2] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (s2 < ns) {
-                    const float* row = po + (size_t)(s2 * rows_max + rl) * ATT_PO_STRIDE;
-                    ml[s2] = *reinterpret_cast<const float2*>(row + HS_HEAD_DIM);
-                    v[s2] = *reinterpret_cast<const float4*>(row + c4 * 4);
-                }
+                if (s2 < ns) ml[s2] = *reinterpret_cast<const float2*>(po + (size_t)(s2 * rows_max + tid) * ATT_PB_STRIDE + HS_HEAD_DIM * 2);
+                Mx = fmaxf(Mx, ml[s2].x);
             }
-            float Mx = -CUDART_INF_F;
-#pragma unroll
-            for (int s2 = 0; s2 < ATT_MAX_SPLIT; ++s2) Mx = fmaxf(Mx, ml[s2].x);
-            float lsum = 0.f;
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            float w[ATT_MAX_SPLIT], lsum = 0.f;
 #pragma unroll
             for (int s2 = 0; s2 < ATT_MAX_SPLIT; ++s2) {
-                const float w = (ml[s2].x == -CUDART_INF_F) ? 0.f : ex2_approx(ml[s2].x - Mx);
-                lsum = fmaf(w, ml[s2].y, lsum);
-                acc.x = fmaf(w, v[s2].x, acc.x); acc.y = fmaf(w, v[s2].y, acc.y);
-                acc.z = fmaf(w, v[s2].z, acc.z); acc.w = fmaf(w, v[s2].w, acc.w);
+                w[s2] = (ml[s2].x == -CUDART_INF_F) ? 0.f : ex2_approx(ml[s2].x - Mx) * ml[s2].y;
+                lsum += w[s2];
+            }
+            const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+#pragma unroll
+            for (int s2 = 0; s2 < ATT_MAX_SPLIT; ++s2) s_wt[tid * ATT_MAX_SPLIT + s2] = w[s2] * inv;
+            const long long og = s_og[tid];
+            if (og >= 0 && p.lse_out) p.lse_out[og] = (Mx + log2f(lsum)) * LN2;
+        }
+        if (tid < UM_SM_THREADS)                             // the softmax threads: the weights are written
+            asm volatile("bar.sync 2, %0;" ::"r"(UM_SM_THREADS) : "memory");
+        // items = (row, 16-byte column group of 8); every item combines one group of each split, all from local shared memory
+        for (int it = tid; it < (r_hi - r_lo) * 16 && tid < UM_SM_THREADS; it += UM_SM_THREADS) {
+            const int rl = it >> 4, c8 = it & 15;
+            float acc[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+#pragma unroll
+            for (int s2 = 0; s2 < ATT_MAX_SPLIT; ++s2) {
+                if (s2 < ns) {
+                    const float w = s_wt[rl * ATT_MAX_SPLIT + s2];
+                    const uint4 v = *reinterpret_cast<const uint4*>(po + (size_t)(s2 * rows_max + rl) * ATT_PB_STRIDE + c8 * 16);
+                    acc[0] = fmaf(w, bf16_lo(v.x), acc[0]); acc[1] = fmaf(w, bf16_hi(v.x), acc[1]);
+                    acc[2] = fmaf(w, bf16_lo(v.y), acc[2]); acc[3] = fmaf(w, bf16_hi(v.y), acc[3]);
+                    acc[4] = fmaf(w, bf16_lo(v.z), acc[4]); acc[5] = fmaf(w, bf16_hi(v.z), acc[5]);
+                    acc[6] = fmaf(w, bf16_lo(v.w), acc[6]); acc[7] = fmaf(w, bf16_hi(v.w), acc[7]);
+                }
             }
             const long long og = s_og[rl];
             if (og >= 0) {
-                const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
-                uint2 packed;
-                packed.x = pack_bf16(acc.x * inv, acc.y * inv);
-                packed.y = pack_bf16(acc.z * inv, acc.w * inv);
-                *reinterpret_cast<uint2*>(p.out + (size_t)og * HS_HEAD_DIM + c4 * 4) = packed;
-                if (p.lse_out && c4 == 0) p.lse_out[og] = (Mx + log2f(lsum)) * LN2;
+                uint4 packed;
+                packed.x = pack_bf16(acc[0], acc[1]); packed.y = pack_bf16(acc[2], acc[3]);
+                packed.z = pack_bf16(acc[4], acc[5]); packed.w = pack_bf16(acc[6], acc[7]);
+                *reinterpret_cast<uint4*>(p.out + (size_t)og * HS_HEAD_DIM + c8 * 8) = packed;
             }
         }
         cluster_wait();
