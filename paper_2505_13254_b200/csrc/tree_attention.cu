@@ -97,7 +97,25 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
 tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV) {
     extern __shared__ unsigned char smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int pair = blockIdx.z, b = pair / p.hkv, h = pair % p.hkv;
+    // Sequences are taken longest prefix first (a ragged batch then ends on its short sequences, not on a long one
+    // that started late): grid slot z / hkv holds the sequence of that rank by (length descending, index ascending).
+    // kv_off is an input of the call, so the ranking runs ahead of the dependency wait.
+    __shared__ int s_seq;
+    int b = blockIdx.z / p.hkv;
+    const int h = blockIdx.z % p.hkv;
+    if (p.batch > 1 && p.batch <= UM_THREADS) {
+        if (tid < p.batch) {
+            const int len = p.kv_off[tid + 1] - p.kv_off[tid];
+            int rank = 0;
+            for (int j = 0; j < p.batch; ++j) {
+                const int lj = p.kv_off[j + 1] - p.kv_off[j];
+                rank += (lj > len || (lj == len && j < tid));
+            }
+            if (rank == b) s_seq = tid;
+        }
+        __syncthreads();
+        b = s_seq;
+    }
     const int split = blockIdx.y;
     const int m0 = blockIdx.x * ATT_BM;
 
