@@ -12,6 +12,7 @@ Steps (one module each):
   attention   tree-masked attention of kept nodes over prefix + tree (Sec. 2.2)
   accept      greedy and rejection-sampling acceptance (Sec. 2.1)
   philox      Philox4x32-10 uniforms (Salmon et al., SC'11), own implementation
+  expand      draft-tree expansion and reranking (Sec. 2.2), the step ahead of verification
 
 Parity pins: every function is pinned by tests/test_oracle_*.py against closed
 forms, invariants, brute force or a published known answer, except the numeric
@@ -19,7 +20,7 @@ values of the seven entropy thresholds, which the paper does not publish
 ("parity unpinned": thresholds are an input here).
 """
 
-from . import accept, attention, philox, row_stats, step, tree  # noqa: F401
+from . import accept, attention, expand, philox, row_stats, step, tree  # noqa: F401
 
 
 def bf16_bits_to_f64(bits):
