@@ -255,6 +255,45 @@ hs_status hs_philox_uniforms(hs_ctx* ctx, uint64_t seed, uint64_t offset, const 
                              const int32_t* node, const int32_t* stream_id, int32_t count,
                              float* out, hs_stream stream);
 
+/* ---- the step ahead of verification: growing and reranking the draft tree ------------------------ */
+
+/* Candidate tree of Sec. 2.2 ("Expansion"), all arrays DEVICE memory owned by the caller.  Sequence b owns slots
+ * b * cap .. b * cap + n_cand[b] - 1 in creation order (candidate 0 = the root, parents precede children).
+ * cap >= 1 + top_k + (levels - 1) * top_k^2 holds a tree of that many levels. */
+typedef struct {
+    int32_t batch;
+    int32_t cap;          /* slots per sequence; hs_rerank takes at most 2048 */
+    int32_t top_k;        /* children per expanded node = width of the frontier, 1 .. HS_MAX_TOPK */
+    int32_t* n_cand;      /* [B] candidates so far */
+    int32_t* parent;      /* [B*cap] candidate id of the parent, -1 for the root */
+    int32_t* token;       /* [B*cap] */
+    int32_t* depth;       /* [B*cap] */
+    float* logc;          /* [B*cap] ln c: log-confidence of the token under its parent's draft row */
+    float* score;         /* [B*cap] ln V_i = sum of logc along the path */
+    int32_t* frontier;    /* [B*top_k] candidates the draft model is run on next, best first */
+    int32_t* n_frontier;  /* [B] */
+    int32_t* status;      /* [B] 0, HS_ERR_SHAPE (cap exhausted) or HS_ERR_BAD_TREE (a row with fewer than top_k finite logits) */
+} hs_expand_state;
+
+/* Sec. 2.2: the tree holds the root only, the frontier is the root. */
+hs_status hs_expand_init(hs_ctx* ctx, const hs_expand_state* st, hs_stream stream);
+
+/* Sec. 2.2 "Expansion", one level (Sec. 4.3: called d' = d_base + Delta times): row b * top_k + j of the three
+ * statistics arrays belongs to the draft row after frontier[b * top_k + j] - exactly what hs_entropy_quantify
+ * writes to topk_val / topk_idx (row stride topk_stride >= top_k, best first) and row_lse for those rows.  Every
+ * frontier node gets its top_k tokens as children (value = parent's + ln c); the top_k children with the
+ * largest value, ties to the one created first, are the next frontier. */
+hs_status hs_expand_level(hs_ctx* ctx, const hs_expand_state* st, const float* topk_val, const int32_t* topk_idx,
+                          const float* row_lse, int32_t topk_stride, hs_stream stream);
+
+/* Sec. 2.2 "Reranking" (Sec. 4.3: with N' in place of N): the n_top[b] (NULL: n_default) candidates with the
+ * largest value, root included, as a tree in creation order: node_off[B+1], and per kept node its parent among
+ * the kept nodes, token, candidate id and depth (arrays of at least sum of min(N, n_cand) entries).  The result is
+ * an hs_tree_batch for the verification calls. */
+hs_status hs_rerank(hs_ctx* ctx, const hs_expand_state* st, const int32_t* n_top, int32_t n_default,
+                    int32_t* node_off, int32_t* parent, int32_t* token, int32_t* cand_id, int32_t* depth,
+                    hs_stream stream);
+
 #ifdef __cplusplus
 }
 #endif

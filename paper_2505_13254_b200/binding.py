@@ -56,6 +56,11 @@ class _AttnDesc(C.Structure):
                 ("kv_head_stride", C.c_int64), ("sm_scale", C.c_float)]
 
 
+class _ExpandState(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("cap", C.c_int32), ("top_k", C.c_int32)] + \
+               [(n, vp) for n in ("n_cand", "parent", "token", "depth", "logc", "score", "frontier", "n_frontier", "status")]
+
+
 class _AcceptOut(C.Structure):
     _fields_ = [(n, vp) for n in ("accept_len", "path_nodes", "path_compact", "path_tokens", "bonus_token",
                                   "terminal_rank", "status")] + [("path_cap", C.c_int32)]
@@ -63,7 +68,8 @@ class _AcceptOut(C.Structure):
 
 EXPORTS = ("hs_status_string", "hs_workspace_bytes", "hs_create", "hs_destroy", "hs_device_error", "hs_entropy_quantify",
            "hs_stratify_prune", "hs_tree_verify_attention", "hs_accept_path", "hs_philox_uniforms",
-           "hs_entropy_quantify_static", "hs_set_prefetch", "hs_selftest_wait_timeout")
+           "hs_entropy_quantify_static", "hs_set_prefetch", "hs_selftest_wait_timeout", "hs_expand_init",
+           "hs_expand_level", "hs_rerank")
 
 
 def lib() -> C.CDLL:
@@ -93,6 +99,9 @@ def lib() -> C.CDLL:
         L.hs_accept_path.argtypes = [C.c_void_p, C.POINTER(_TreeBatch), C.POINTER(_PrunedTree), vp, C.c_int32, vp,
                                      C.c_int, C.c_int64, C.c_int32, vp, vp, C.c_uint64, C.c_uint64, vp,
                                      C.POINTER(_AcceptOut), vp]
+        L.hs_expand_init.argtypes = [C.c_void_p, C.POINTER(_ExpandState), vp]
+        L.hs_expand_level.argtypes = [C.c_void_p, C.POINTER(_ExpandState), vp, vp, vp, C.c_int32, vp]
+        L.hs_rerank.argtypes = [C.c_void_p, C.POINTER(_ExpandState), vp, C.c_int32, vp, vp, vp, vp, vp, vp]
         L.hs_philox_uniforms.argtypes = [C.c_void_p, C.c_uint64, C.c_uint64, vp, vp, vp, C.c_int32, vp, vp]
         for name in EXPORTS:
             if name not in ("hs_status_string", "hs_workspace_bytes"):
@@ -325,3 +334,41 @@ def hs_philox_uniforms(ctx: Context, seed: int, offset: int, b: torch.Tensor, no
     _check(lib().hs_philox_uniforms(ctx.handle, seed, offset, _ptr(b), _ptr(node), _ptr(stream_id), b.numel(),
                                     _ptr(out), _stream()), "hs_philox_uniforms")
     return out
+
+
+class ExpandState(_Bundle):
+    """Device arrays of the candidate tree (hs_expand_state)."""
+    _cstruct = _ExpandState
+
+    def __init__(self, batch: int, cap: int, top_k: int, device):
+        i = lambda *s: torch.zeros(*s, dtype=torch.int32, device=device)
+        f = lambda *s: torch.zeros(*s, dtype=torch.float32, device=device)
+        self.batch, self.cap, self.top_k = batch, cap, top_k
+        self.n_cand, self.n_frontier, self.status = i(batch), i(batch), i(batch)
+        self.parent, self.token, self.depth = i(batch, cap), i(batch, cap), i(batch, cap)
+        self.logc, self.score = f(batch, cap), f(batch, cap)
+        self.frontier = i(batch, top_k)
+
+
+def hs_expand_init(ctx: Context, st: ExpandState) -> None:
+    c = st.c()
+    _check(lib().hs_expand_init(ctx.handle, C.byref(c), _stream()), "hs_expand_init")
+
+
+def hs_expand_level(ctx: Context, st: ExpandState, quant: QuantOut) -> None:
+    """One expansion level from the row statistics of the frontier rows (row b * top_k + j = frontier j of b)."""
+    c = st.c()
+    _check(lib().hs_expand_level(ctx.handle, C.byref(c), _ptr(quant.topk_val), _ptr(quant.topk_idx),
+                                 _ptr(quant.row_lse), quant.topk_val.shape[1], _stream()), "hs_expand_level")
+
+
+def hs_rerank(ctx: Context, st: ExpandState, n_top: Optional[torch.Tensor], n_default: int):
+    """Returns (node_off, parent, token, cand_id, depth): the reranked trees as one CSR batch."""
+    dev = st.parent.device
+    rows = st.batch * min(st.cap, max(n_default, int(n_top.max()) if n_top is not None else 0))
+    i = lambda *s: torch.zeros(*s, dtype=torch.int32, device=dev)
+    node_off, parent, token, cand_id, depth = i(st.batch + 1), i(rows), i(rows), i(rows), i(rows)
+    c = st.c()
+    _check(lib().hs_rerank(ctx.handle, C.byref(c), _ptr(n_top), n_default, _ptr(node_off), _ptr(parent), _ptr(token),
+                           _ptr(cand_id), _ptr(depth), _stream()), "hs_rerank")
+    return node_off, parent, token, cand_id, depth
