@@ -294,6 +294,20 @@ hs_status hs_rerank(hs_ctx* ctx, const hs_expand_state* st, const int32_t* n_top
                     int32_t* node_off, int32_t* parent, int32_t* token, int32_t* cand_id, int32_t* depth,
                     hs_stream stream);
 
+/* ---- training of the stratifier ------------------------------------------------------------------- */
+
+/* Sec. 4.2, Eq. 2: CART regression on one feature.  x[n] = Phi(P*) of n verified trees (phi_star of
+ * hs_entropy_quantify), y[n] = their Terminal Confidence Rank (terminal_rank of hs_accept_path, as floats), both
+ * DEVICE arrays.  Every layer splits every node at the threshold s that minimises
+ *   L(s) = sum over {left, right} of |D_j| / |D| * sum over D_j of (y - mean_j)^2
+ * over the midpoints between consecutive distinct feature values (ties: the smallest s).  thresholds (device,
+ * 2^depth - 1 floats) receives the thresholds in ascending order: with depth = 3 they are hs_policy.thresholds.
+ * status (device, one int): 0, or HS_ERR_SHAPE if some node held a single feature value (its threshold is NaN).
+ * 1 <= depth <= 6, 2^depth <= n <= 2^26.  Needs hs_cart_workspace_bytes(n) of context workspace. */
+size_t hs_cart_workspace_bytes(int32_t n);
+hs_status hs_cart_fit(hs_ctx* ctx, const float* x, const float* y, int32_t n, int32_t depth, float* thresholds,
+                      int32_t* status, hs_stream stream);
+
 #ifdef __cplusplus
 }
 #endif

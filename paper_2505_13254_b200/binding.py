@@ -69,7 +69,7 @@ class _AcceptOut(C.Structure):
 EXPORTS = ("hs_status_string", "hs_workspace_bytes", "hs_create", "hs_destroy", "hs_device_error", "hs_entropy_quantify",
            "hs_stratify_prune", "hs_tree_verify_attention", "hs_accept_path", "hs_philox_uniforms",
            "hs_entropy_quantify_static", "hs_set_prefetch", "hs_selftest_wait_timeout", "hs_expand_init",
-           "hs_expand_level", "hs_rerank")
+           "hs_expand_level", "hs_rerank", "hs_cart_fit", "hs_cart_workspace_bytes")
 
 
 def lib() -> C.CDLL:
@@ -102,9 +102,12 @@ def lib() -> C.CDLL:
         L.hs_expand_init.argtypes = [C.c_void_p, C.POINTER(_ExpandState), vp]
         L.hs_expand_level.argtypes = [C.c_void_p, C.POINTER(_ExpandState), vp, vp, vp, C.c_int32, vp]
         L.hs_rerank.argtypes = [C.c_void_p, C.POINTER(_ExpandState), vp, C.c_int32, vp, vp, vp, vp, vp, vp]
+        L.hs_cart_workspace_bytes.restype = C.c_size_t
+        L.hs_cart_workspace_bytes.argtypes = [C.c_int32]
+        L.hs_cart_fit.argtypes = [C.c_void_p, vp, vp, C.c_int32, C.c_int32, vp, vp, vp]
         L.hs_philox_uniforms.argtypes = [C.c_void_p, C.c_uint64, C.c_uint64, vp, vp, vp, C.c_int32, vp, vp]
         for name in EXPORTS:
-            if name not in ("hs_status_string", "hs_workspace_bytes"):
+            if name not in ("hs_status_string", "hs_workspace_bytes", "hs_cart_workspace_bytes"):
                 getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -372,3 +375,16 @@ def hs_rerank(ctx: Context, st: ExpandState, n_top: Optional[torch.Tensor], n_de
     _check(lib().hs_rerank(ctx.handle, C.byref(c), _ptr(n_top), n_default, _ptr(node_off), _ptr(parent), _ptr(token),
                            _ptr(cand_id), _ptr(depth), _stream()), "hs_rerank")
     return node_off, parent, token, cand_id, depth
+
+
+def hs_cart_workspace_bytes(n: int) -> int:
+    return int(lib().hs_cart_workspace_bytes(n))
+
+
+def hs_cart_fit(ctx: Context, x: torch.Tensor, y: torch.Tensor, depth: int = 3):
+    """Trains the stratifier on (Phi(P*), Terminal Confidence Rank) pairs.  Returns (thresholds [2^depth - 1], status [1])."""
+    th = torch.empty((1 << depth) - 1, dtype=torch.float32, device=x.device)
+    status = torch.zeros(1, dtype=torch.int32, device=x.device)
+    _check(lib().hs_cart_fit(ctx.handle, _ptr(x), _ptr(y), x.numel(), depth, _ptr(th), _ptr(status), _stream()),
+           "hs_cart_fit")
+    return th, status

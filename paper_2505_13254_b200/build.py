@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libheterospec.so")
-SOURCES = ["hs_api.cu", "row_stats.cu", "stratify_prune.cu", "tree_attention.cu", "accept.cu", "expand.cu"]
+SOURCES = ["hs_api.cu", "row_stats.cu", "stratify_prune.cu", "tree_attention.cu", "accept.cu", "expand.cu", "cart.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 
