@@ -221,6 +221,18 @@ hs_status hs_entropy_quantify_static(const hs_tree_batch* tree, const void* draf
 hs_status hs_stratify_prune(hs_ctx* ctx, const hs_tree_batch* tree, const hs_quant_out* quant,
                             const hs_policy* policy, const hs_pruned_tree* out, hs_stream stream);
 
+/* hs_stratify_prune under a token budget (App. A.8: "hardware budget", the tokens one forward pass of the target
+ * model may process, shared by the batch).  The paper names the goal - Top-N pruning frees budget on low-entropy
+ * requests, which is handed to requests with stricter service-level objectives - but no algorithm; this call
+ * implements: every sequence first asks for min(N', nodes of depth <= d'); if the requests fit `budget`, the
+ * tokens left over go to the sequences in order of slo_class[b] (device [B]; smaller = stricter = served first,
+ * ties by sequence index), each up to its nodes of depth <= d'; otherwise the excess is taken back in the
+ * opposite order, never below the root.  The reallocated counts replace N' in the Top-N reranking (n_keep
+ * reports them, n_prime still the policy's N'); the sum of n_keep is at most max(budget, B). */
+hs_status hs_stratify_prune_budget(hs_ctx* ctx, const hs_tree_batch* tree, const hs_quant_out* quant,
+                                   const hs_policy* policy, const int32_t* slo_class, int32_t budget,
+                                   const hs_pruned_tree* out, hs_stream stream);
+
 /* Sec. 2.2 tree-mask attention.  q, out: [rows][hq][128] bf16; k_tree, v_tree: [rows][hkv][128]
  * bf16 (keys/values of the kept tree tokens, already position-encoded); k_cache, v_cache: bf16
  * with the strides of `desc`; lse_out (nullable): [rows][hq] float, natural-log normaliser.

@@ -69,7 +69,7 @@ class _AcceptOut(C.Structure):
 EXPORTS = ("hs_status_string", "hs_workspace_bytes", "hs_create", "hs_destroy", "hs_device_error", "hs_entropy_quantify",
            "hs_stratify_prune", "hs_tree_verify_attention", "hs_accept_path", "hs_philox_uniforms",
            "hs_entropy_quantify_static", "hs_set_prefetch", "hs_selftest_wait_timeout", "hs_expand_init",
-           "hs_expand_level", "hs_rerank", "hs_cart_fit", "hs_cart_workspace_bytes")
+           "hs_expand_level", "hs_rerank", "hs_cart_fit", "hs_cart_workspace_bytes", "hs_stratify_prune_budget")
 
 
 def lib() -> C.CDLL:
@@ -94,6 +94,8 @@ def lib() -> C.CDLL:
                                                  C.POINTER(_Policy), C.POINTER(_QuantOut), vp]
         L.hs_stratify_prune.argtypes = [C.c_void_p, C.POINTER(_TreeBatch), C.POINTER(_QuantOut),
                                         C.POINTER(_Policy), C.POINTER(_PrunedTree), vp]
+        L.hs_stratify_prune_budget.argtypes = [C.c_void_p, C.POINTER(_TreeBatch), C.POINTER(_QuantOut),
+                                               C.POINTER(_Policy), vp, C.c_int32, C.POINTER(_PrunedTree), vp]
         L.hs_tree_verify_attention.argtypes = [C.c_void_p, C.POINTER(_PrunedTree), C.POINTER(_AttnDesc), vp, vp, vp,
                                                vp, vp, vp, vp, vp]
         L.hs_accept_path.argtypes = [C.c_void_p, C.POINTER(_TreeBatch), C.POINTER(_PrunedTree), vp, C.c_int32, vp,
@@ -289,6 +291,16 @@ def hs_stratify_prune(ctx: Context, tree: TreeBatch, quant: QuantOut, policy: di
     t, q, p, o = tree.c(), quant.c(), make_policy(policy), out.c()
     _check(lib().hs_stratify_prune(ctx.handle, C.byref(t), C.byref(q), C.byref(p), C.byref(o), _stream()),
            "hs_stratify_prune")
+    return out
+
+
+def hs_stratify_prune_budget(ctx: Context, tree: TreeBatch, quant: QuantOut, policy: dict, slo_class: torch.Tensor,
+                             budget: int, out: Optional[PrunedTree] = None) -> PrunedTree:
+    if out is None:
+        out = PrunedTree(tree.n_nodes_total, tree.batch, tree.parent.device)
+    t, q, p, o = tree.c(), quant.c(), make_policy(policy), out.c()
+    _check(lib().hs_stratify_prune_budget(ctx.handle, C.byref(t), C.byref(q), C.byref(p), _ptr(slo_class), budget,
+                                          C.byref(o), _stream()), "hs_stratify_prune_budget")
     return out
 
 

@@ -169,6 +169,18 @@ extern "C" hs_status hs_stratify_prune(hs_ctx* ctx, const hs_tree_batch* tree, c
     return hs_launch_stratify_prune(ctx, tree, quant, policy, out, (cudaStream_t)stream);
 }
 
+extern "C" hs_status hs_stratify_prune_budget(hs_ctx* ctx, const hs_tree_batch* tree, const hs_quant_out* quant,
+                                              const hs_policy* policy, const int32_t* slo_class, int32_t budget,
+                                              const hs_pruned_tree* out, hs_stream stream) {
+    if (!ctx || !quant || !out || !slo_class || budget < 0 || !hs_on_device(ctx)) return HS_ERR_INVALID_ARG;
+    if (!tree_ok(tree) || !policy_ok(policy)) return HS_ERR_INVALID_ARG;
+    if (!quant->score || !quant->phi_star || !quant->depth || !quant->status) return HS_ERR_INVALID_ARG;
+    if (!out->bin || !out->d_prime || !out->n_prime || !out->n_keep || !out->keep_off || !out->keep_idx ||
+        !out->new_parent || !out->new_depth || !out->keep_rank || !out->anc_mask || !out->status)
+        return HS_ERR_INVALID_ARG;
+    return hs_launch_stratify_prune_budget(ctx, tree, quant, policy, slo_class, budget, out, (cudaStream_t)stream);
+}
+
 static bool pruned_ok(const hs_pruned_tree* p) {
     return p && p->n_keep && p->keep_off && p->keep_idx && p->new_parent && p->new_depth && p->keep_rank &&
            p->anc_mask && p->status;

@@ -158,6 +158,9 @@ hs_status hs_launch_quantify(hs_ctx* ctx, const hs_tree_batch* tree, const void*
                              const hs_quant_out* out, cudaStream_t stream);
 hs_status hs_launch_stratify_prune(hs_ctx* ctx, const hs_tree_batch* tree, const hs_quant_out* quant,
                                    const hs_policy* policy, const hs_pruned_tree* out, cudaStream_t stream);
+hs_status hs_launch_stratify_prune_budget(hs_ctx* ctx, const hs_tree_batch* tree, const hs_quant_out* quant,
+                                          const hs_policy* policy, const int32_t* slo_class, int32_t budget,
+                                          const hs_pruned_tree* out, cudaStream_t stream);
 hs_status hs_launch_attention(hs_ctx* ctx, const hs_pruned_tree* pruned, const hs_attn_desc* desc,
                               const void* q, const void* k_tree, const void* v_tree, const void* k_cache,
                               const void* v_cache, void* out, float* lse_out, cudaStream_t stream);

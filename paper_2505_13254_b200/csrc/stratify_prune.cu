@@ -20,7 +20,12 @@ struct PruneParams {
     const int* depth;
     const int* qstatus;
     hs_pruned_tree out;
-    int counted;           // out.n_keep was filled by prune_count_kernel
+    int counted;           // out.n_keep was filled by a launch ahead (prune_count_kernel or budget_kernel)
+    const int* n_override; // [B] node counts that replace the policy's N' (budget reallocation), or NULL
+    int* base;             // [B] budget path: policy request min(N', eligible), 0 for a flagged sequence
+    int* room;             // [B] budget path: eligible nodes
+    const int* slo_class;  // [B] budget path
+    int budget;
     float th[7];
     int d_base, alpha, n_default, gamma_pct[3];
 };
@@ -68,6 +73,113 @@ __global__ void __launch_bounds__(128) prune_count_kernel(const PruneParams p) {
         cnt = max(0, min(np, elig));
     }
     if (lane == 0) p.out.n_keep[b] = cnt;
+}
+
+// budget path, first launch: one warp per sequence, the policy's request and the eligible nodes
+__global__ void __launch_bounds__(128) budget_request_kernel(const PruneParams p) {
+    const int lane = threadIdx.x & 31;
+    const int b = blockIdx.x * 4 + (threadIdx.x >> 5);
+    pdl_launch_dependents();
+    pdl_wait();
+    if (b >= p.batch) return;
+    int base = 0, elig = 0;
+    if (p.qstatus[b] == 0) {
+        int bin, dp, np;
+        policy_lookup(p, p.phi_star[b], bin, dp, np);
+        const int lo = p.node_off[b], hi = min(p.node_off[b + 1], lo + HS_MAX_NODES);
+        for (int i = lo + lane; i < hi; i += 32) elig += (p.depth[i] <= dp);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) elig += __shfl_xor_sync(HS_FULL_MASK, elig, o);
+        elig = max(elig, 1);
+        base = max(1, min(np, elig));
+    }
+    if (lane == 0) { p.base[b] = base; p.room[b] = elig; }
+}
+
+// budget path, second launch (one CTA): App. A.8 reading - if the requests fit the budget the left-over tokens go to
+// the sequences in order of SLO class (stricter first, then sequence index), each up to its eligible nodes;
+// otherwise the excess is taken back in the opposite order, never below the root.  The order is found by a
+// bitonic sort of (class, index) keys in shared memory, the hand-out by a running sum along that order.
+#define BUDGET_THREADS 1024
+__global__ void __launch_bounds__(BUDGET_THREADS) budget_kernel(const PruneParams p) {
+    __shared__ unsigned int s_key[HS_MAX_BATCH];
+    __shared__ int s_amt[HS_MAX_BATCH];          // what the sequence at a sorted position may take (or give back)
+    __shared__ int s_red[BUDGET_THREADS / 32];
+    __shared__ int s_total;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pdl_launch_dependents();
+    pdl_wait();
+    const int B = p.batch;
+    int P = 32;
+    while (P < B) P <<= 1;
+    int part = 0;
+    for (int b = tid; b < B; b += BUDGET_THREADS) part += p.base[b];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(HS_FULL_MASK, part, o);
+    if (lane == 0) s_red[warp] = part;
+    __syncthreads();
+    if (tid == 0) {
+        int t = 0;
+        for (int w = 0; w < BUDGET_THREADS / 32; ++w) t += s_red[w];
+        s_total = t;
+    }
+    __syncthreads();
+    const int total = s_total;
+    const bool fits = total <= p.budget;
+    // keys: ascending = order of service; over budget the order is reversed (loosest class, highest index first)
+    for (int i = tid; i < P; i += BUDGET_THREADS) {
+        unsigned int k = 0xffffffffu;
+        if (i < B) {
+            const unsigned int cls = (unsigned int)min(max(p.slo_class[i], 0), 0xffff);
+            k = (cls << 16) | (unsigned int)i;
+            if (!fits) k = 0xfffffffeu - k;
+        }
+        s_key[i] = k;
+    }
+    __syncthreads();
+    for (int k = 2; k <= P; k <<= 1)
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int t = tid; t < P / 2; t += BUDGET_THREADS) {
+                const int i = 2 * t - (t & (j - 1));
+                const bool up = (i & k) == 0;
+                const unsigned int a = s_key[i], c = s_key[i + j];
+                if ((a > c) == up) { s_key[i] = c; s_key[i + j] = a; }
+            }
+            __syncthreads();
+        }
+    auto seq_of = [&](int pos) -> int {
+        unsigned int k = s_key[pos];
+        if (k == 0xffffffffu) return -1;
+        if (!fits) k = 0xfffffffeu - k;
+        return (int)(k & 0xffffu);
+    };
+    for (int pos = tid; pos < P; pos += BUDGET_THREADS) {
+        const int b = seq_of(pos);
+        int a = 0;
+        if (b >= 0 && p.base[b] > 0) a = fits ? p.room[b] - p.base[b] : p.base[b] - 1;
+        s_amt[pos] = a;
+    }
+    __syncthreads();
+    // the amount still to hand out (or take back) when the walk reaches a position = pool - sum of the amounts ahead
+    const int pool = fits ? p.budget - total : total - p.budget;
+    const int per = (P + BUDGET_THREADS - 1) / BUDGET_THREADS;          // consecutive positions per thread
+    int mine = 0;
+    for (int q = 0; q < per; ++q) { const int pos = tid * per + q; if (pos < P) mine += s_amt[pos]; }
+    int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int u = __shfl_up_sync(HS_FULL_MASK, incl, o); if (lane >= o) incl += u; }
+    if (lane == 31) s_red[warp] = incl;
+    __syncthreads();
+    int before = incl - mine;
+    for (int w = 0; w < warp; ++w) before += s_red[w];
+    for (int q = 0; q < per; ++q) {
+        const int pos = tid * per + q;
+        if (pos >= P) break;
+        const int b = seq_of(pos);
+        const int take = max(0, min(s_amt[pos], pool - before));
+        before += s_amt[pos];
+        if (b >= 0) p.out.n_keep[b] = p.base[b] == 0 ? 0 : (fits ? p.base[b] + take : p.base[b] - take);
+    }
 }
 
 __global__ void __launch_bounds__(HS_MAX_NODES) stratify_prune_kernel(const PruneParams p) {
@@ -122,7 +234,7 @@ __global__ void __launch_bounds__(HS_MAX_NODES) stratify_prune_kernel(const Prun
         for (int j = 0; j < n; ++j)
             rank += (s_elig[j] && (s_S[j] > S || (s_S[j] == S && j < tid)));
     }
-    const bool keep = elig && rank < np;
+    const bool keep = elig && rank < (p.n_override ? p.n_override[b] : np);
     // compaction: ballot inside the warp, prefix over the four warps
     const unsigned int bal = __ballot_sync(HS_FULL_MASK, keep);
     __syncthreads();                       // s_warp is reused
@@ -178,9 +290,42 @@ hs_status hs_launch_stratify_prune(hs_ctx* ctx, const hs_tree_batch* tree, const
     p.alpha = policy->alpha;
     p.n_default = policy->n_default;
     for (int i = 0; i < 3; ++i) p.gamma_pct[i] = policy->gamma_pct[i];
+    p.n_override = nullptr; p.base = nullptr; p.room = nullptr; p.slo_class = nullptr; p.budget = 0;
     p.counted = p.batch > 32;
     if (p.counted &&
         hs_launch(prune_count_kernel, dim3((p.batch + 3) / 4), dim3(128), 0, stream, ctx->pdl, dim3(1, 1, 1), p) != cudaSuccess)
+        return HS_ERR_CUDA;
+    return hs_launch(stratify_prune_kernel, dim3(p.batch), dim3(HS_MAX_NODES), 0, stream, ctx->pdl, dim3(1, 1, 1), p) ==
+                   cudaSuccess ? HS_OK : HS_ERR_CUDA;
+}
+
+// Sec. 4.2-4.3 with the token budget of App. A.8: request -> reallocation -> Top-N reranking with the reallocated counts.
+hs_status hs_launch_stratify_prune_budget(hs_ctx* ctx, const hs_tree_batch* tree, const hs_quant_out* quant,
+                                          const hs_policy* policy, const int32_t* slo_class, int32_t budget,
+                                          const hs_pruned_tree* out, cudaStream_t stream) {
+    PruneParams p;
+    p.batch = tree->batch;
+    p.node_off = tree->node_off;
+    p.parent = tree->parent;
+    p.score = quant->score;
+    p.phi_star = quant->phi_star;
+    p.depth = quant->depth;
+    p.qstatus = quant->status;
+    p.out = *out;
+    for (int i = 0; i < 7; ++i) p.th[i] = policy->thresholds[i];
+    p.d_base = policy->d_base;
+    p.alpha = policy->alpha;
+    p.n_default = policy->n_default;
+    for (int i = 0; i < 3; ++i) p.gamma_pct[i] = policy->gamma_pct[i];
+    if ((size_t)2 * p.batch * sizeof(int) > ctx->scratch_bytes) return HS_ERR_WORKSPACE;
+    p.base = (int*)ctx->scratch;
+    p.room = p.base + p.batch;
+    p.slo_class = slo_class;
+    p.budget = budget;
+    p.counted = 1;
+    p.n_override = out->n_keep;
+    if (hs_launch(budget_request_kernel, dim3((p.batch + 3) / 4), dim3(128), 0, stream, ctx->pdl, dim3(1, 1, 1), p) != cudaSuccess ||
+        hs_launch(budget_kernel, dim3(1), dim3(BUDGET_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p) != cudaSuccess)
         return HS_ERR_CUDA;
     return hs_launch(stratify_prune_kernel, dim3(p.batch), dim3(HS_MAX_NODES), 0, stream, ctx->pdl, dim3(1, 1, 1), p) ==
                    cudaSuccess ? HS_OK : HS_ERR_CUDA;
