@@ -188,6 +188,7 @@ typedef struct {
     int32_t* terminal_rank;/* [B] confidence rank of the terminal node (Terminal Confidence Rank) */
     int32_t* status;       /* [B] */
     int32_t path_cap;      /* slots per sequence, > deepest kept node */
+    int32_t max_kept_rows; /* host: upper bound of the kept nodes of the whole batch, 0 = n_nodes_total; sizes the grid */
 } hs_accept_out;
 
 /* ---- the four steps ----------------------------------------------------------------------- */

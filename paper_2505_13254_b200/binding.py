@@ -63,7 +63,7 @@ class _ExpandState(C.Structure):
 
 class _AcceptOut(C.Structure):
     _fields_ = [(n, vp) for n in ("accept_len", "path_nodes", "path_compact", "path_tokens", "bonus_token",
-                                  "terminal_rank", "status")] + [("path_cap", C.c_int32)]
+                                  "terminal_rank", "status")] + [("path_cap", C.c_int32), ("max_kept_rows", C.c_int32)]
 
 
 EXPORTS = ("hs_status_string", "hs_workspace_bytes", "hs_create", "hs_destroy", "hs_device_error", "hs_entropy_quantify",
@@ -243,6 +243,7 @@ class AcceptOut(_Bundle):
         self.accept_len, self.bonus_token, self.terminal_rank, self.status = i(batch), i(batch), i(batch), i(batch)
         self.path_nodes, self.path_compact, self.path_tokens = i(batch, path_cap), i(batch, path_cap), i(batch, path_cap)
         self.path_cap = path_cap
+        self.max_kept_rows = 0
 
 
 def _dtype_code(t: torch.Tensor) -> int:

@@ -799,7 +799,8 @@ hs_status hs_launch_accept(hs_ctx* ctx, const hs_tree_batch* tree, const hs_prun
     p.offset = offset;
     p.uniforms = uniforms;
     p.out = *out;
-    const int rows = tree->n_nodes_total;          // upper bound of kept nodes
+    int rows = tree->n_nodes_total;                // upper bound of kept nodes
+    if (out->max_kept_rows > 0 && out->max_kept_rows < rows) rows = out->max_kept_rows;
     size_t o = 0;
     p.ro.tgt_arg = (int*)(ctx->scratch + o); o += hs_align_up((size_t)rows * sizeof(int), 256);
     p.ro.tgt_ms = (float2*)(ctx->scratch + o); o += hs_align_up((size_t)rows * sizeof(float2), 256);

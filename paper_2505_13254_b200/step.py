@@ -85,9 +85,9 @@ class VerifyStep:
     def prune(self, db: DeviceBatch):
         return hb.hs_stratify_prune(self.ctx, db.tree, self.quant, self.policy, out=self.pruned)
 
-    def attention(self, db: DeviceBatch):
+    def attention(self, db: DeviceBatch, max_nodes: Optional[int] = None):
         return hb.hs_tree_verify_attention(self.ctx, self.pruned, db.q, db.k_tree, db.v_tree, db.k_cache, db.v_cache,
-                                           db.kv_off, batch=db.tree.batch, max_nodes=db.max_nodes,
+                                           db.kv_off, batch=db.tree.batch, max_nodes=max_nodes or db.max_nodes,
                                            max_kv_len=db.max_kv_len, layout=hb.HS_ROWS_ORIGINAL,
                                            node_off=db.tree.node_off, out=self.attn_out, lse_out=self.attn_lse)
 
@@ -139,4 +139,58 @@ class GraphedStep:
 
     def replay(self) -> VerifyStep:
         self.graph.replay()
+        return self.step
+
+
+def regime_bounds(policy: dict, max_nodes: int):
+    """The kept-node bounds of the regimes of Sec. 4.3: N' of the three low-entropy bins and of the others, ascending,
+    capped by the drafted tree size."""
+    b = set()
+    for i in range(3):
+        delta = policy["alpha"] - i
+        b.add(min(max_nodes, (policy["gamma_pct"][i] * policy["n_default"] + 50) // 100 + delta))
+    b.add(min(max_nodes, policy["n_default"]))
+    b.add(max_nodes)
+    return sorted(b)
+
+
+class RegimeStep:
+    """Sec. 4.3, Dynamic Computational Adaptation: a computation graph kept ready per regime.  The step runs in two
+    phases: graph 1 = quantify + stratify/prune, after which the host reads the largest kept-node count of the
+    batch (four bytes: the host has to know it anyway, it is the token count of the target model's forward pass);
+    graph 2 = tree attention + acceptance, one graph per regime, captured with grids sized to that regime's N'
+    instead of the drafted tree.  A regime is keyed by its bound on the kept nodes per sequence."""
+
+    def __init__(self, step: VerifyStep, db: DeviceBatch, warmup: int = 2):
+        self.step, self.db = step, db
+        self.n_keep_host = torch.zeros(1, dtype=torch.int32).pin_memory()
+        self.n_keep_max = torch.zeros(1, dtype=torch.int32, device=db.tree.parent.device)
+        for _ in range(warmup):
+            step.run(db)
+        torch.cuda.synchronize()
+        self.phase1 = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.phase1):
+            step.quantify(db)
+            step.prune(db)
+            torch.amax(step.pruned.n_keep, dim=0, keepdim=True, out=self.n_keep_max)
+            self.n_keep_host.copy_(self.n_keep_max, non_blocking=True)
+        self.bounds = regime_bounds(step.policy, db.max_nodes)
+        self.phase2 = {}
+        for bound in self.bounds:
+            step.accept.max_kept_rows = min(db.tree.n_nodes_total, bound * db.tree.batch)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                if db.q is not None:
+                    step.attention(db, max_nodes=bound)
+                step.accept_path(db)
+            self.phase2[bound] = g
+        step.accept.max_kept_rows = 0
+        self.last_bound = None
+
+    def replay(self) -> VerifyStep:
+        self.phase1.replay()
+        torch.cuda.current_stream().synchronize()            # the host learns the regime
+        n = int(self.n_keep_host[0])
+        self.last_bound = next(b for b in self.bounds if b >= n)
+        self.phase2[self.last_bound].replay()
         return self.step

@@ -39,3 +39,4 @@ def test_struct_sizes_match_the_header():
     assert ctypes.sizeof(binding._TreeBatch) == 8 + 3 * 8
     assert ctypes.sizeof(binding._AttnDesc) == 9 * 4 + 4 + 2 * 8 + 2 * 8 + 8
     assert ctypes.sizeof(binding._AcceptOut) == 7 * 8 + 8
+    assert ctypes.sizeof(binding._ExpandState) == 3 * 4 + 4 + 9 * 8

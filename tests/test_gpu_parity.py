@@ -133,3 +133,30 @@ def test_graph_replay_across_bins(ctx):
         pu.check_attention(st.attn_out, st.attn_lse, batch, res)
         pu.check_accept(st.accept, res)
         assert hb.hs_device_error(ctx) == 0
+
+
+# ---- a graph per regime, grids sized to the regime's N' (Sec. 4.3, Dynamic Computational Adaptation) ---------------------
+
+def test_regime_graphs_across_bins(ctx):
+    cfg, base = SMALL["c2_small"]
+    policy = pu.policy_for(cfg, base)
+    cases = [pu.oracle_case(cfg, policy, seed) for seed in (2100, 2200, 2300, 2400, 2500, 2600)]
+    db = gstep.upload(cases[0][0])
+    st = gstep.VerifyStep(ctx, db, policy)
+    rs = gstep.RegimeStep(st, db)
+    assert rs.bounds == [22, 39, 60]                       # N' of bins 0, 1 and of the rest (62 is capped by the 60 drafted nodes)
+    used = set()
+    for batch, res in cases[1:] + cases[:1]:
+        batch = dict(batch, philox_seed=cases[0][0]["philox_seed"], philox_offset=cases[0][0]["philox_offset"])
+        gstep.refill(db, batch)
+        rs.replay()
+        torch.cuda.synchronize()
+        nk = len(res[0]["pruned"]["keep_idx"])
+        assert rs.last_bound == min(b for b in rs.bounds if b >= nk)
+        used.add(rs.last_bound)
+        pu.check_quant(st.quant, batch, res, policy["top_k"])
+        pu.check_pruned(st.pruned, res)
+        pu.check_attention(st.attn_out, st.attn_lse, batch, res)
+        pu.check_accept(st.accept, res)
+        assert hb.hs_device_error(ctx) == 0
+    assert len(used) >= 2                                  # the seeds land in regimes with different graphs
