@@ -416,6 +416,30 @@ def main():
                                       "traffic": ncu_traffic("tree_attn_umma_kernel", cfg.name),
                                       "algorithmic_bytes_per_launch": attn_bytes,
                                       "algorithmic_flops_per_launch": attn_flops}
+    # ---- a graph per regime (Sec. 4.3): the same tree forced into the lowest and into the highest entropy bin ---------
+    if world == 1:
+        regimes = {}
+        for name, th in (("bin0", 1e9), ("bin7", -1e9)):
+            pol = dict(policy, thresholds=[th] * 7)
+            st_r = gstep.VerifyStep(ctx, db0, pol)
+            rs = gstep.RegimeStep(st_r, db0)
+            one = gstep.GraphedStep(st_r, db0)
+            n_rep = min(args.steps, 300)
+
+            def wall(fn):
+                for _ in range(5):
+                    fn()
+                torch.cuda.synchronize()
+                t = time.perf_counter()
+                for _ in range(n_rep):
+                    fn()
+                torch.cuda.synchronize()
+                return 1e6 * (time.perf_counter() - t) / n_rep
+            regimes[name] = {"kept_nodes": int(st_r.pruned.n_keep.sum().item()), "graph_bound": rs.last_bound,
+                             "two_phase_us": wall(rs.replay), "one_graph_us": wall(one.replay)}
+        line["regime_graphs"] = dict(regimes, how="wall clock per step over back-to-back replays on one input copy (L2-warm); "
+                                     "two_phase = quantify + prune, the host reads the kept-node count, then the regime's own "
+                                     "graph of attention + acceptance; one_graph = all calls in one graph sized by the drafted tree")
     if not args.no_cpu_baseline:
         from oracle import step as ostep
         nrep = 5

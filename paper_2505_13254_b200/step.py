@@ -186,6 +186,7 @@ class RegimeStep:
             self.phase2[bound] = g
         step.accept.max_kept_rows = 0
         self.last_bound = None
+        self.replay()                                        # (sets last_bound; results of the warm-up batch)
 
     def replay(self) -> VerifyStep:
         self.phase1.replay()
