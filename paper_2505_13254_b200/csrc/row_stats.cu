@@ -5,7 +5,7 @@
 //     items of up to 32 KiB (bulk copies into a ring of shared-memory slots, completion on mbarriers); sixteen
 //     consumer warps reduce each item in ONE pass: running maximum per thread (packed bf16 maxima), then
 //     sum e^(x-m) and sum x e^(x-m) with the exponent's multiply-add and the two sums as packed fp32 pairs.
-//     Top-K without sorting: after every window of three items a warp takes a lower bound of the K-th
+//     Top-K without sorting: after the first items of a row share a warp takes a lower bound of the K-th
 //     largest logit of the row share from maxima of disjoint element sets (the 32 half-warp maxima of the
 //     CTA, or its own 32 lane maxima on a short share), and only lanes whose window maximum reaches the bound
 //     re-scan their vectors in shared memory and push candidates; the few candidates are ranked by counting.
@@ -32,7 +32,7 @@
 #define QS_ITEM_VECS 2048                     // vectors per item: 32 KiB, four per consumer thread
 #define QS_VPT (QS_ITEM_VECS / QS_CONSUMERS)
 #define QS_SLOTS 6                            // ring of item slots
-#define QS_WINDOW 3                           // items a consumer holds before it hands their slots back
+#define QS_WINDOW 4                           // items a consumer holds before it hands their slots back
 #define QS_MAX_SEGS 32                        // shares a row may be split over
 #define QS_SMEM_BYTES (QS_SLOTS * QS_ITEM_VECS * 16 + 128)
 
@@ -542,9 +542,12 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
                 if (lane < HS_MAX_TOPK) p.part_keys[(size_t)ps * HS_MAX_TOPK + lane] = (lane < K) ? top[lane] : 0ull;
                 __syncwarp();
                 if (lane == 0) {
-                    __threadfence();
-                    const int last = atomicAdd(&p.row_cnt[row], 1) == nseg - 1;
-                    if (last) { p.row_cnt[row] = 0; __threadfence(); }     // (counter ready for the next launch)
+                    // one release-acquire arrival at device scope: the partial written by this warp (ordered before the
+                    // arrival by the warp barrier above) is visible to whoever arrives last, and the last one sees all
+                    int old;
+                    asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(old) : "l"(&p.row_cnt[row]) : "memory");
+                    const int last = old == nseg - 1;
+                    if (last) p.row_cnt[row] = 0;              // ready for the next launch
                     s_flag = last;
                 }
             }
