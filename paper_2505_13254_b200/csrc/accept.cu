@@ -616,7 +616,7 @@ __device__ int cluster_inverse_cdf(const AcceptParams& p, cg::cluster_group& clu
     return pick != 0x7fffffff ? pick : max(lastp, 0);
 }
 
-__global__ void __cluster_dims__(WALK_CLUSTER, 1, 1) __launch_bounds__(WALK_THREADS)
+__global__ void __cluster_dims__(WALK_CLUSTER, 1, 1) __launch_bounds__(WALK_THREADS, 1)
 accept_walk_kernel(const AcceptParams p) {
     cg::cluster_group cluster = cg::this_cluster();
     extern __shared__ __align__(16) unsigned char s_rows[];    // staged: this CTA's slices of p and q, `per` vectors each
@@ -692,21 +692,48 @@ accept_walk_kernel(const AcceptParams p) {
         rs.p = (const uint4*)s_rows;
         rs.q = qrow ? (const uint4*)s_rows + per : nullptr;
     };
+    // Every candidate's probability under its parent's target and draft row, its uniform and the normalisers of its
+    // own rows, for all kept nodes at once (three dependent round trips in all instead of three per visited node);
+    // the walk below then runs from shared memory until a rejection needs a vocabulary-wide residual sum.  Every CTA
+    // of the cluster fetches the same values and takes the same decisions.
+    __shared__ int s_par[HS_MAX_NODES], s_tok[HS_MAX_NODES], s_orig[HS_MAX_NODES];
+    __shared__ float s_pt[HS_MAX_NODES], s_qt[HS_MAX_NODES], s_u[HS_MAX_NODES];
+    __shared__ float2 s_pms[HS_MAX_NODES];
+    const float T = p.temperature[b];
+    const float invT = LOG2E / T;
+    const int nkc = min(nk, HS_MAX_NODES);
+    for (int j = tid; j < nkc; j += WALK_THREADS) {
+        const int par = p.pr.new_parent[koff + j];
+        const int orig = p.pr.keep_idx[koff + j];
+        const int tok = p.token[nbase + orig];
+        s_par[j] = par; s_tok[j] = tok; s_orig[j] = orig;
+        s_pms[j] = p.ro.tgt_ms[koff + j];
+        float pt = 0.f, qt = 0.f;
+        if (par >= 0 && par < nkc) {
+            const int porig = p.pr.keep_idx[koff + par];
+            const int trow = p.target_layout == HS_ROWS_ORIGINAL ? nbase + porig : koff + par;
+            const char* prow = (const char*)p.target + (size_t)trow * p.row_stride * esz;
+            const char* qrow = (const char*)p.draft + (size_t)(nbase + porig) * p.row_stride * esz;
+            const float2 pms = p.ro.tgt_ms[koff + par], qms = p.ro.drf_ms[koff + par];
+            pt = exp2f((fmaxf(load_logit(prow, p.is_bf16, tok), -1e30f) - pms.x) * invT) * (1.f / pms.y);
+            qt = exp2f((fmaxf(load_logit(qrow, p.is_bf16, tok), -1e30f) - qms.x) * invT) * (1.f / qms.y);
+        }
+        s_pt[j] = pt; s_qt[j] = qt;
+        s_u[j] = p.uniforms ? p.uniforms[nbase + orig] : philox_uniform(p.seed, p.offset, b, orig, 0);
+    }
     __syncthreads();
     int cur = 0, len = 0, bonus = -1;
     {
-        const float T = p.temperature[b];
-        const float invT = LOG2E / T;
-        for (int step = 0; step < nk; ++step) {
+        for (int step = 0; step < nkc; ++step) {
             if (rank == 0 && tid == 0 && len < cap) {
                 p.out.path_compact[b * cap + len] = cur;
-                p.out.path_nodes[b * cap + len] = p.pr.keep_idx[koff + cur];
+                p.out.path_nodes[b * cap + len] = s_orig[cur];
             }
-            const int trow = p.target_layout == HS_ROWS_ORIGINAL ? nbase + p.pr.keep_idx[koff + cur] : koff + cur;
-            const int drow = nbase + p.pr.keep_idx[koff + cur];
+            const int trow = p.target_layout == HS_ROWS_ORIGINAL ? nbase + s_orig[cur] : koff + cur;
+            const int drow = nbase + s_orig[cur];
             const char* prow = (const char*)p.target + (size_t)trow * p.row_stride * esz;
             const char* qrow = (const char*)p.draft + (size_t)drow * p.row_stride * esz;
-            const float2 pms = p.ro.tgt_ms[koff + cur];
+            const float2 pms = s_pms[cur];
             const float pm = pms.x, ips = 1.f / pms.y;
             float qm = 0.f, iqs = 0.f;
             bool have_q = false;
@@ -714,21 +741,31 @@ accept_walk_kernel(const AcceptParams p) {
             double W = 1.0;
             int accepted = -1;
             bool tested = false;
-            for (int j = cur + 1; j < nk; ++j) {                 // siblings in index order
-                if (p.pr.new_parent[koff + j] != cur) continue;
+            // the kept children of cur as bit masks (every warp finds them with four ballots instead of a serial scan)
+            unsigned int kids[HS_MAX_NODES / 32];
+#pragma unroll
+            for (int w = 0; w < HS_MAX_NODES / 32; ++w) {
+                const int j = w * 32 + (tid & 31);
+                kids[w] = __ballot_sync(HS_FULL_MASK, j > cur && j < nkc && s_par[j] == cur);
+            }
+            for (;;) {                                           // siblings in index order
+                int j = -1;
+#pragma unroll
+                for (int w = HS_MAX_NODES / 32 - 1; w >= 0; --w)
+                    if (kids[w]) j = w * 32 + __ffs(kids[w]) - 1;
+                if (j < 0) break;
+#pragma unroll
+                for (int w = 0; w < HS_MAX_NODES / 32; ++w)
+                    if (j >> 5 == w) kids[w] &= kids[w] - 1;
+                tested = true;
+                const float pt = s_pt[j], qt = s_qt[j];
+                const float r = fmaxf(pt - c * qt, 0.f) / (float)W;
+                const float a = qt > 0.f ? fminf(1.f, r / qt) : 1.f;
+                if (s_u[j] < a) { accepted = j; break; }
                 if (!have_q) {
                     const float2 qms = p.ro.drf_ms[koff + cur];
                     qm = qms.x; iqs = 1.f / qms.y; have_q = true;
                 }
-                tested = true;
-                const int orig = p.pr.keep_idx[koff + j];
-                const int t = p.token[nbase + orig];
-                const float pt = exp2f((fmaxf(load_logit(prow, p.is_bf16, t), -1e30f) - pm) * invT) * ips;
-                const float qt = exp2f((fmaxf(load_logit(qrow, p.is_bf16, t), -1e30f) - qm) * invT) * iqs;
-                const float r = fmaxf(pt - c * qt, 0.f) / (float)W;
-                const float a = qt > 0.f ? fminf(1.f, r / qt) : 1.f;
-                const float u = p.uniforms ? p.uniforms[nbase + orig] : philox_uniform(p.seed, p.offset, b, orig, 0);
-                if (u < a) { accepted = j; break; }
                 const float c_next = c + (float)W;
                 stage(cur, prow, qrow);
                 const double W_next = cluster_residual_sum(p, cluster, rs, pm, ips, qm, iqs, invT,
@@ -737,8 +774,7 @@ accept_walk_kernel(const AcceptParams p) {
                 c = c_next; W = W_next;
             }
             if (accepted >= 0) {
-                if (rank == 0 && tid == 0 && len < cap)
-                    p.out.path_tokens[b * cap + len] = p.token[nbase + p.pr.keep_idx[koff + accepted]];
+                if (rank == 0 && tid == 0 && len < cap) p.out.path_tokens[b * cap + len] = s_tok[accepted];
                 cur = accepted;
                 ++len;
                 continue;
