@@ -504,17 +504,30 @@ struct RowSlice {
     int v0, nv;
 };
 
+// All-gather of one 64-bit value per CTA over the cluster: warp 0 of every CTA stores its value into slot `rank` of the
+// exchange buffer of all WALK_CLUSTER CTAs (posted stores through distributed shared memory, lane r to CTA r), one
+// cluster barrier makes them visible, every CTA then reads its own copy.  The buffers alternate from one exchange to
+// the next (s_x[xch & 1]), so one barrier per exchange is enough: a buffer is written again only two exchanges later,
+// after a barrier that every CTA reaches with its reads done.  `v` must be valid in warp 0.
+__device__ __forceinline__ void cluster_allgather(unsigned long long v, unsigned long long (*s_x)[WALK_CLUSTER],
+                                                  unsigned int& xch, unsigned int rank) {
+    unsigned long long* buf = s_x[xch & 1u];
+    ++xch;
+    if (threadIdx.x < WALK_CLUSTER) {
+        const unsigned int remote = cluster_map_addr(smem_u32(&buf[rank]), threadIdx.x);
+        asm volatile("st.shared::cluster.b64 [%0], %1;" ::"r"(remote), "l"(v) : "memory");
+    }
+    cluster_arrive();
+    cluster_wait();
+}
+
 // Sum over this CTA's share of the vocabulary of max(p_v - c q_v, 0), then over the cluster.
-// Every CTA returns the same value (fixed summation order).  The CTAs' sums are exchanged through s_cta[xch & 1]:
-// the buffers alternate from one exchange to the next, so one cluster barrier per exchange is enough (a buffer is
-// written again only two exchanges later, after a barrier that every CTA reaches with its reads done).
-__device__ double cluster_residual_sum(const AcceptParams& p, cg::cluster_group& cluster, const RowSlice& rs,
+// Every CTA returns the same value (fixed summation order).
+__device__ double cluster_residual_sum(const AcceptParams& p, unsigned int rank, const RowSlice& rs,
                                        float pm, float ips, float qm, float iqs, float invT,
-                                       float c, double* s_part, double* s_cta2, unsigned int& xch) {
+                                       float c, double* s_part, unsigned long long (*s_x)[WALK_CLUSTER], unsigned int& xch) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int ve = p.is_bf16 ? 8 : 4;
-    double* s_cta = s_cta2 + (xch & 1u);
-    ++xch;
     float acc = 0.f;
     for (int v = tid; v < rs.nv; v += WALK_THREADS) {
         uint4 a = rs.p[v], bq = rs.q[v];
@@ -532,27 +545,25 @@ __device__ double cluster_residual_sum(const AcceptParams& p, cg::cluster_group&
     double w = warp_sum_d((double)acc);
     if (lane == 0) s_part[warp] = w;
     __syncthreads();
-    if (tid == 0) {
-        double t = 0.0;
+    double t = 0.0;
+    if (warp == 0) {                                   // the warps' sums in a fixed order, known to every lane of warp 0
         for (int i = 0; i < WALK_THREADS / 32; ++i) t += s_part[i];
-        *s_cta = t;
     }
-    cluster.sync();
+    const unsigned long long* got = s_x[xch & 1u];
+    cluster_allgather((unsigned long long)__double_as_longlong(t), s_x, xch, rank);
     double tot = 0.0;
-    for (unsigned int r = 0; r < WALK_CLUSTER; ++r) tot += *cluster.map_shared_rank(s_cta, r);
+    for (unsigned int r = 0; r < WALK_CLUSTER; ++r) tot += __longlong_as_double((long long)got[r]);
     return tot;
 }
 
 // Inverse-CDF draw from max(p - c q, 0) in token order: smallest j whose running sum exceeds
 // u * total; if rounding leaves none, the last token with positive mass.  rs.q may be NULL (c = 0).
 // A CTA covers the tokens of its slice, a thread a contiguous run of them; running sums in double.
-__device__ int cluster_inverse_cdf(const AcceptParams& p, cg::cluster_group& cluster, const RowSlice& rs,
+__device__ int cluster_inverse_cdf(const AcceptParams& p, unsigned int rank, const RowSlice& rs,
                                    float pm, float ips, float qm, float iqs, float invT,
-                                   float c, float u, double* s_scan, double* s_cta2, unsigned int& xch, int* s_pick) {
+                                   float c, float u, double* s_scan, unsigned long long (*s_x)[WALK_CLUSTER],
+                                   unsigned int& xch, int* s_pick) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const unsigned int rank = cluster.block_rank();
-    double* s_cta = s_cta2 + (xch & 1u);
-    ++xch;
     const int ve = p.is_bf16 ? 8 : 4;
     const int c0 = rs.v0 * ve, c1 = min(c0 + rs.nv * ve, p.vocab);
     const int seg = (max(c1 - c0, 0) + WALK_THREADS - 1) / WALK_THREADS;
@@ -587,11 +598,11 @@ __device__ int cluster_inverse_cdf(const AcceptParams& p, cg::cluster_group& clu
         if (w < warp) wbefore += t;
         ctot += t;
     }
-    if (tid == 0) *s_cta = ctot;
-    cluster.sync();
+    const unsigned long long* got = s_x[xch & 1u];
+    cluster_allgather((unsigned long long)__double_as_longlong(ctot), s_x, xch, rank);
     double before = 0.0, total = 0.0;
     for (unsigned int r = 0; r < WALK_CLUSTER; ++r) {
-        double v = *cluster.map_shared_rank(s_cta, r);
+        const double v = __longlong_as_double((long long)got[r]);
         if (r < rank) before += v;
         total += v;
     }
@@ -605,14 +616,15 @@ __device__ int cluster_inverse_cdf(const AcceptParams& p, cg::cluster_group& clu
     }
     if (last_pos >= 0) atomicMax(&s_pick[1], last_pos);
     __syncthreads();
-    cluster.sync();
+    // the CTAs' (crossing, last positive token) pairs, one 64-bit word each
+    const unsigned long long mine2 = ((unsigned long long)(unsigned int)s_pick[0] << 32) | (unsigned int)s_pick[1];
+    const unsigned long long* got2 = s_x[xch & 1u];
+    cluster_allgather(mine2, s_x, xch, rank);
     int pick = 0x7fffffff, lastp = -1;
     for (unsigned int r = 0; r < WALK_CLUSTER; ++r) {
-        const int* sp = cluster.map_shared_rank(s_pick, r);
-        pick = min(pick, sp[0]);
-        lastp = max(lastp, sp[1]);
+        pick = min(pick, (int)(unsigned int)(got2[r] >> 32));
+        lastp = max(lastp, (int)(unsigned int)(got2[r] & 0xffffffffu));
     }
-    cluster.sync();
     return pick != 0x7fffffff ? pick : max(lastp, 0);
 }
 
@@ -623,7 +635,7 @@ accept_walk_kernel(const AcceptParams p) {
     __shared__ unsigned long long s_bar;
     __shared__ double s_part[WALK_THREADS / 32];
     __shared__ double s_scan[WALK_THREADS / 32];
-    __shared__ double s_cta[2];
+    __shared__ unsigned long long s_x[2][WALK_CLUSTER];    // all-gather buffers of the cluster exchanges
     unsigned int xch = 0;                  // exchanges through s_cta so far
     __shared__ int s_pick[2];
     __shared__ int s_child;
@@ -768,8 +780,8 @@ accept_walk_kernel(const AcceptParams p) {
                 }
                 const float c_next = c + (float)W;
                 stage(cur, prow, qrow);
-                const double W_next = cluster_residual_sum(p, cluster, rs, pm, ips, qm, iqs, invT,
-                                                           c_next, s_part, s_cta, xch);
+                const double W_next = cluster_residual_sum(p, rank, rs, pm, ips, qm, iqs, invT,
+                                                           c_next, s_part, s_x, xch);
                 if (!(W_next > 0.0)) { c = 0.f; W = 1.0; tested = false; break; }   // p == q: fall back to p
                 c = c_next; W = W_next;
             }
@@ -781,11 +793,12 @@ accept_walk_kernel(const AcceptParams p) {
             }
             const float ufin = p.uniforms ? p.uniforms[p.n_nodes_total + b] : philox_uniform(p.seed, p.offset, b, 0, 1);
             stage(cur, prow, (tested && c > 0.f) ? qrow : nullptr);
-            bonus = cluster_inverse_cdf(p, cluster, rs, pm, ips, qm, iqs,
-                                        invT, c, ufin, s_scan, s_cta, xch, s_pick);
+            bonus = cluster_inverse_cdf(p, rank, rs, pm, ips, qm, iqs,
+                                        invT, c, ufin, s_scan, s_x, xch, s_pick);
             break;
         }
     }
+    // (every store into a CTA's exchange buffers precedes a barrier that CTA takes part in: it may leave now)
     if (rank == 0 && tid == 0) {
         p.out.accept_len[b] = len;
         p.out.bonus_token[b] = bonus;
