@@ -534,8 +534,9 @@ __device__ double cluster_residual_sum(const AcceptParams& p, unsigned int rank,
         float x[8], y[8];
         if (p.is_bf16) { unpack_v<true>(a, x); unpack_v<true>(bq, y); }
         else { unpack_v<false>(a, x); unpack_v<false>(bq, y); }
-        for (int e = 0; e < ve; ++e) {
-            if ((rs.v0 + v) * ve + e < p.vocab) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            if (e < ve && (rs.v0 + v) * ve + e < p.vocab) {
                 float pv = exp2f((fmaxf(x[e], -1e30f) - pm) * invT) * ips;
                 float qv = exp2f((fmaxf(y[e], -1e30f) - qm) * invT) * iqs;
                 acc += fmaxf(pv - c * qv, 0.f);
