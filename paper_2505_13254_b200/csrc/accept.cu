@@ -78,45 +78,47 @@ __device__ __forceinline__ void unpack_v(const uint4& v, float* x) {
 // child whose token is the arg-max of the current node's target row until no child matches; the bonus
 // token is the arg-max where the walk stops.  tgt_arg was written by other CTAs: read it past L1.
 __device__ void greedy_walk(const AcceptParams& p, int b) {
-    __shared__ int s_child;
+    __shared__ int s_arg[HS_MAX_NODES], s_next[HS_MAX_NODES], s_orig[HS_MAX_NODES];
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int koff = p.pr.keep_off[b];
-    const int nk = p.pr.n_keep[b];
+    const int nk = min(p.pr.n_keep[b], HS_MAX_NODES);
     const int nbase = p.node_off[b];
     const int cap = p.out.path_cap;
+    // Every kept node's parent, token and its row's arg-max in one round trip; the walk itself then runs in shared
+    // memory: node j continues the path of its parent iff its token is the parent's arg-max, and of several such
+    // children (duplicate tokens among siblings) the one with the lowest index does.
+    int my_par = -1, my_tok = -1;
+    if (tid < nk) {
+        my_par = p.pr.new_parent[koff + tid];
+        const int orig = p.pr.keep_idx[koff + tid];
+        s_arg[tid] = __ldcg(&p.ro.tgt_arg[koff + tid]);
+        s_orig[tid] = orig;
+        s_next[tid] = 0x7fffffff;
+        my_tok = p.token[nbase + orig];
+    }
     for (int j = tid; j < cap; j += nthr) {
         p.out.path_nodes[b * cap + j] = -1;
         p.out.path_compact[b * cap + j] = -1;
         p.out.path_tokens[b * cap + j] = -1;
     }
     __syncthreads();
-    // this thread's kept nodes: parent and token stay in registers for the whole walk (nk <= 128 <= nthr)
-    int my_par = -2, my_tok = -1;
-    if (tid < nk) {
-        my_par = p.pr.new_parent[koff + tid];
-        my_tok = p.token[nbase + p.pr.keep_idx[koff + tid]];
-    }
-    int cur = 0, len = 0, bonus = -1;
-    for (int step = 0; step < nk; ++step) {
-        const int g = __ldcg(&p.ro.tgt_arg[koff + cur]);
-        if (tid == 0) s_child = 0x7fffffff;
-        __syncthreads();
-        if (tid > cur && my_par == cur && my_tok == g) atomicMin(&s_child, tid);
-        __syncthreads();
-        const int nxt = s_child;
-        __syncthreads();
-        if (tid == 0 && len < cap) {
-            p.out.path_compact[b * cap + len] = cur;
-            p.out.path_nodes[b * cap + len] = p.pr.keep_idx[koff + cur];
-        }
-        if (nxt == 0x7fffffff) { bonus = g; break; }
-        if (tid == 0 && len < cap) p.out.path_tokens[b * cap + len] = g;
-        cur = nxt;
-        ++len;
-    }
+    if (tid > 0 && tid < nk && my_par >= 0 && my_par < tid && my_tok == s_arg[my_par]) atomicMin(&s_next[my_par], tid);
+    __syncthreads();
     if (tid == 0) {
+        int cur = 0, len = 0;
+        for (int step = 0; step < nk; ++step) {
+            if (len < cap) {
+                p.out.path_compact[b * cap + len] = cur;
+                p.out.path_nodes[b * cap + len] = s_orig[cur];
+            }
+            const int nxt = s_next[cur];
+            if (nxt == 0x7fffffff) break;
+            if (len < cap) p.out.path_tokens[b * cap + len] = s_arg[cur];
+            cur = nxt;
+            ++len;
+        }
         p.out.accept_len[b] = len;
-        p.out.bonus_token[b] = bonus;
+        p.out.bonus_token[b] = s_arg[cur];
         p.out.terminal_rank[b] = p.pr.keep_rank[koff + cur];
         p.out.status[b] = HS_OK;
     }
@@ -428,14 +430,16 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 4) accept_rows_kernel(const __
         }
         p.partials[((size_t)which * p.part_rows + k) * p.chunks + chunk] =
             make_uint4((unsigned int)best, (unsigned int)(best >> 32), __float_as_uint(M), __float_as_uint(S));
-        __threadfence();
+        // one release-acquire arrival at device scope: this thread's partial is visible to whoever arrives last,
+        // and the last one (then, behind the barrier below, its whole CTA) sees all of them
         int* cnt = &p.row_cnt[which * HS_MAX_ROWS + k];
-        s_flag = (atomicAdd(cnt, 1) == p.chunks - 1);
+        int old;
+        asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(old) : "l"(cnt) : "memory");
+        s_flag = (old == p.chunks - 1);
         if (s_flag) *cnt = 0;
     }
     __syncthreads();
     if (!s_flag) return;
-    __threadfence();
     if (warp == 0) {
     // last chunk of the row: merge (chunks <= 32, one lane per chunk)
     unsigned long long ck = 0ull;
@@ -477,11 +481,11 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 4) accept_rows_kernel(const __
     }
     if (which != 0 || md == HS_ACCEPT_REJECTION) return;
     __syncthreads();
-    if (tid == 0) {
-        __threadfence();
-        s_flag = (atomicAdd(&p.seq_cnt[b], 1) == nk - 1);
+    if (tid == 0) {                                // (the thread that wrote the row's merged result)
+        int old;
+        asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(old) : "l"(&p.seq_cnt[b]) : "memory");
+        s_flag = (old == nk - 1);
         if (s_flag) p.seq_cnt[b] = 0;
-        __threadfence();
     }
     __syncthreads();
     if (s_flag) {
