@@ -94,6 +94,16 @@ hs_status hs_destroy(hs_ctx* ctx);
 #define HS_PREFETCH_KV 2       /* k_cache / v_cache of hs_tree_verify_attention */
 hs_status hs_set_prefetch(hs_ctx* ctx, int32_t flags);
 
+/* Which kernel hs_accept_path reads the vocabulary rows with (a tuning knob; the paper has no counterpart).  Both give
+ * the same results.  HS_ROW_PASS_CHUNK: one small CTA per 32 KiB of a row, all loads in flight at once - shortest
+ * latency when the rows of a step are few.  HS_ROW_PASS_STREAM: one persistent CTA per SM with a producer warp and
+ * a ring of shared-memory slots - highest bandwidth when the rows of a step exceed what is in flight at once.
+ * HS_ROW_PASS_AUTO (default): the stream from 48 MiB of rows (upper bound of kept rows x row bytes), else chunks. */
+#define HS_ROW_PASS_AUTO 0
+#define HS_ROW_PASS_CHUNK 1
+#define HS_ROW_PASS_STREAM 2
+hs_status hs_set_row_pass(hs_ctx* ctx, int32_t variant);
+
 /* Reads and clears the context's sticky device error word into *host_out (host pointer): HS_OK, or
  * HS_ERR_TIMEOUT if a kernel gave up a bounded wait since the last call.  Synchronises the device. */
 hs_status hs_device_error(hs_ctx* ctx, int32_t* host_out);

@@ -20,6 +20,7 @@ HS_F32, HS_BF16 = 0, 1
 HS_ACCEPT_GREEDY, HS_ACCEPT_REJECTION, HS_ACCEPT_DETERMINISTIC = 0, 1, 2
 HS_ROWS_COMPACT, HS_ROWS_ORIGINAL = 0, 1
 HS_PREFETCH_LOGITS, HS_PREFETCH_KV = 1, 2
+HS_ROW_PASS_AUTO, HS_ROW_PASS_CHUNK, HS_ROW_PASS_STREAM = 0, 1, 2
 HS_ERR_INVALID_ARG, HS_ERR_SHAPE, HS_ERR_WORKSPACE, HS_ERR_TIMEOUT, HS_ERR_BAD_TREE = 1, 2, 4, 6, 7
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libheterospec.so")
@@ -68,7 +69,7 @@ class _AcceptOut(C.Structure):
 
 EXPORTS = ("hs_status_string", "hs_workspace_bytes", "hs_create", "hs_destroy", "hs_device_error", "hs_entropy_quantify",
            "hs_stratify_prune", "hs_tree_verify_attention", "hs_accept_path", "hs_philox_uniforms",
-           "hs_entropy_quantify_static", "hs_set_prefetch", "hs_selftest_wait_timeout", "hs_expand_init",
+           "hs_entropy_quantify_static", "hs_set_prefetch", "hs_set_row_pass", "hs_selftest_wait_timeout", "hs_expand_init",
            "hs_expand_level", "hs_rerank", "hs_cart_fit", "hs_cart_workspace_bytes", "hs_stratify_prune_budget")
 
 
@@ -87,6 +88,7 @@ def lib() -> C.CDLL:
         L.hs_destroy.argtypes = [C.c_void_p]
         L.hs_device_error.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
         L.hs_set_prefetch.argtypes = [C.c_void_p, C.c_int32]
+        L.hs_set_row_pass.argtypes = [C.c_void_p, C.c_int32]
         L.hs_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_uint64, vp]
         L.hs_entropy_quantify.argtypes = [C.c_void_p, C.POINTER(_TreeBatch), vp, C.c_int, C.c_int64, C.c_int32,
                                           C.POINTER(_Policy), C.POINTER(_QuantOut), vp]
@@ -142,6 +144,10 @@ def hs_device_error(ctx: "Context") -> int:
 
 def hs_set_prefetch(ctx: "Context", flags: int) -> None:
     _check(lib().hs_set_prefetch(ctx.handle, flags), "hs_set_prefetch")
+
+
+def hs_set_row_pass(ctx: "Context", variant: int) -> None:
+    _check(lib().hs_set_row_pass(ctx.handle, variant), "hs_set_row_pass")
 
 
 def hs_selftest_wait_timeout(ctx: "Context", limit_ns: int) -> None:

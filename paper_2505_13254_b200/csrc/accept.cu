@@ -77,9 +77,13 @@ __device__ __forceinline__ void unpack_v(const uint4& v, float* x) {
 // Greedy acceptance of sequence b by one whole CTA (Sec. 5, temperature 0): from the root, move to the kept
 // child whose token is the arg-max of the current node's target row until no child matches; the bonus
 // token is the arg-max where the walk stops.  tgt_arg was written by other CTAs: read it past L1.
+// The two walks below are run by the first HS_ROW_THREADS threads of a CTA (the whole CTA of the chunk kernel, half
+// of the consumer warps of the streaming kernel), which meet on a barrier of their own.
+__device__ __forceinline__ void walk_sync() { named_bar_sync(2, HS_ROW_THREADS); }
+
 __device__ void greedy_walk(const AcceptParams& p, int b) {
     __shared__ int s_arg[HS_MAX_NODES], s_next[HS_MAX_NODES], s_orig[HS_MAX_NODES];
-    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int tid = threadIdx.x, nthr = HS_ROW_THREADS;
     const int koff = p.pr.keep_off[b];
     const int nk = min(p.pr.n_keep[b], HS_MAX_NODES);
     const int nbase = p.node_off[b];
@@ -101,9 +105,9 @@ __device__ void greedy_walk(const AcceptParams& p, int b) {
         p.out.path_compact[b * cap + j] = -1;
         p.out.path_tokens[b * cap + j] = -1;
     }
-    __syncthreads();
+    walk_sync();
     if (tid > 0 && tid < nk && my_par >= 0 && my_par < tid && my_tok == s_arg[my_par]) atomicMin(&s_next[my_par], tid);
-    __syncthreads();
+    walk_sync();
     if (tid == 0) {
         int cur = 0, len = 0;
         for (int step = 0; step < nk; ++step) {
@@ -138,7 +142,7 @@ __device__ __noinline__ void deterministic_walk(const AcceptParams& p, int b) {
     __shared__ double s_phase[64];
     __shared__ double s_wp[64][HS_ROW_THREADS / 32];     // per (phase, warp) sums of pass 1
     __shared__ int s_pick[2];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = HS_ROW_THREADS;
     const int koff = p.pr.keep_off[b];
     const int nk = min(p.pr.n_keep[b], HS_MAX_NODES);
     const int nbase = p.node_off[b];
@@ -152,7 +156,7 @@ __device__ __noinline__ void deterministic_walk(const AcceptParams& p, int b) {
         s_par[j] = p.pr.new_parent[koff + j];
         s_tok[j] = p.token[nbase + p.pr.keep_idx[koff + j]];
     }
-    __syncthreads();
+    walk_sync();
     const float invT = LOG2E / p.temperature[b];
     const size_t esz = p.is_bf16 ? 2 : 4;
     // every candidate's probability under its parent's target row and its uniform, all nodes at once (one round
@@ -170,7 +174,7 @@ __device__ __noinline__ void deterministic_walk(const AcceptParams& p, int b) {
         s_pt[j] = pt;
         s_u[j] = p.uniforms ? p.uniforms[nbase + orig] : philox_uniform(p.seed, p.offset, b, orig, 0);
     }
-    __syncthreads();
+    walk_sync();
     int cur = 0, len = 0, bonus = -1;
     for (int step = 0; step < nk; ++step) {
         if (tid == 0 && len < cap) {
@@ -194,9 +198,9 @@ __device__ __noinline__ void deterministic_walk(const AcceptParams& p, int b) {
             if (s_u[j] < a) { accepted = j; break; }
             const double W_next = W - (double)pt;
             if (!(W_next > 0.0)) { nrej = 0; W = 1.0; break; }  // nothing left: fall back to p
-            __syncthreads();                                     // (every thread walks the same way)
+            walk_sync();                                     // (every thread walks the same way)
             if (tid == 0) s_rej[nrej] = t;
-            __syncthreads();
+            walk_sync();
             ++nrej;
             W = W_next;
         }
@@ -212,7 +216,7 @@ __device__ __noinline__ void deterministic_walk(const AcceptParams& p, int b) {
         // every phase; then the phase that holds the crossing is summed again and scanned.
         const float ufin = p.uniforms ? p.uniforms[p.n_nodes_total + b] : philox_uniform(p.seed, p.offset, b, 0, 1);
         if (tid == 0) { s_pick[0] = 0x7fffffff; s_pick[1] = -1; }
-        __syncthreads();                                         // s_rej, s_pick
+        walk_sync();                                         // s_rej, s_pick
         const int ve = p.is_bf16 ? 8 : 4;
         const int phase_vecs = nthr * 4;
         // (at most 64 phases: the launcher refuses vocabularies of more than 32 chunks = 64 phases)
@@ -262,13 +266,13 @@ __device__ __noinline__ void deterministic_walk(const AcceptParams& p, int b) {
             const double w = warp_sum_d(mine);
             if (lane == 0) s_wp[ph][warp] = w;           // (no barrier per phase: the loads of the next one go out)
         }
-        __syncthreads();
+        walk_sync();
         for (int ph = tid; ph < nph; ph += nthr) {
             double t = 0.0;
             for (int w2 = 0; w2 < nthr / 32; ++w2) t += s_wp[ph][w2];
             s_phase[ph] = t;
         }
-        __syncthreads();
+        walk_sync();
         double total = 0.0;
         for (int ph = 0; ph < nph; ++ph) total += s_phase[ph];
         const double goal = (double)ufin * total;
@@ -293,7 +297,7 @@ __device__ __noinline__ void deterministic_walk(const AcceptParams& p, int b) {
                 if (lane >= o) incl += up;
             }
             if (lane == 31) s_scan[warp] = incl;
-            __syncthreads();
+            walk_sync();
             double run = before_ph + (incl - mine);
             for (int w2 = 0; w2 < warp; ++w2) run += s_scan[w2];
             if (run <= goal && run + mine > goal) {              // the crossing lies in this thread's tokens
@@ -311,7 +315,7 @@ __device__ __noinline__ void deterministic_walk(const AcceptParams& p, int b) {
             }
         }
         if (last_pos >= 0) atomicMax(&s_pick[1], last_pos);
-        __syncthreads();
+        walk_sync();
         bonus = s_pick[0] != 0x7fffffff ? s_pick[0] : max(s_pick[1], 0);
         break;
     }
@@ -491,6 +495,419 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 4) accept_rows_kernel(const __
     if (s_flag) {
         if (md == HS_ACCEPT_GREEDY) greedy_walk(p, b);
         else deterministic_walk(p, b);
+    }
+}
+
+// ================================================================================================================
+// The row pass as a stream (launches whose rows do not fit the latency-bound regime of the chunk kernel)
+// ================================================================================================================
+// The rows to read - the target row of every kept node, then the draft row of every kept internal node of a
+// sequence in rejection mode - form one stream of 16-byte vectors that is cut into equal contiguous shares, one per
+// CTA, one CTA per SM.  Which rows those are is only known on the device (the pruned tree comes from the kernel
+// ahead), so every CTA derives the list itself: a bit per kept node for "needs its draft row", a prefix of the bit
+// counts, the share bounds from the total.  A producer warp looks the rows of the share up (32 at a time, one per
+// lane) and brings them on chip in items of up to 32 KiB (bulk copies into a ring of shared-memory slots); sixteen
+// consumer warps reduce each item in one pass: arg-max with the lowest index on ties (packed bf16 maxima with a
+// 16-bit position code per half-lane, decoded once per row segment) and, for sampling sequences, max and
+// sum e^((x-max)/T).  A row that lies in several shares leaves partials; the last share to arrive merges them.
+// Sequences that finish in the row pass (greedy, deterministic proposals) are walked after the CTA's share by the
+// CTA that merged their last target row.
+#define AS_CONSUMERS 512
+#define AS_NW (AS_CONSUMERS / 32)
+#define AS_THREADS (AS_CONSUMERS + 32)
+#define AS_ITEM_VECS 2048
+#define AS_VPT (AS_ITEM_VECS / AS_CONSUMERS)
+#define AS_SLOTS 5
+#define AS_MAX_SEGS 32
+#define AS_ROW_RING 64
+#define AS_SMEM_BYTES (AS_SLOTS * AS_ITEM_VECS * 16 + 128)
+#define AS_MIN_BYTES ((size_t)48 << 20)       // smaller launches go to the chunk kernel
+
+struct WorkRow {          // one row of the stream, as looked up by the producer warp
+    const char* ptr;
+    int k;                // kept node (index into the compacted arrays)
+    int b;                // its sequence
+    int which;            // 0 target row, 1 draft row
+    int mode;
+    float invT;           // log2(e) / temperature
+    int nk;               // kept nodes of the sequence
+};
+
+template <bool BF16>
+__global__ void __launch_bounds__(AS_THREADS, 1) accept_stream_kernel(const __grid_constant__ AcceptParams p) {
+    constexpr int VE = BF16 ? 8 : 4;
+    constexpr int NWORDS = HS_MAX_ROWS / 32;
+    extern __shared__ __align__(128) unsigned char s_dyn[];
+    __shared__ unsigned long long s_full[AS_SLOTS], s_empty[AS_SLOTS];
+    __shared__ unsigned int s_bits[NWORDS];          // kept node -> its draft row is part of the stream
+    __shared__ int s_pref[NWORDS + 1];               // set bits ahead of each word
+    __shared__ WorkRow s_rows[AS_ROW_RING];
+    __shared__ unsigned long long s_wkey[2][AS_NW];
+    __shared__ float2 s_wms[2][AS_NW];
+    __shared__ unsigned short s_pending[HS_MAX_BATCH];   // sequences this CTA has to walk
+    __shared__ int s_npending;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const unsigned int slots0 = (smem_u32(s_dyn) + 127u) & ~127u;
+    const unsigned char* slots_gen = s_dyn + (slots0 - smem_u32(s_dyn));
+    const size_t esz = BF16 ? 2 : 4;
+
+    if (tid == 0) {
+        for (int s = 0; s < AS_SLOTS; ++s) {
+            mbar_init(smem_u32(&s_full[s]), 1);
+            mbar_init(smem_u32(&s_empty[s]), AS_NW);
+        }
+        mbar_init_fence();
+        s_npending = 0;
+    }
+    for (int i = tid; i < NWORDS; i += AS_THREADS) s_bits[i] = 0u;
+    __syncthreads();
+    pdl_launch_dependents();
+    pdl_wait();                            // the pruned tree and the logits come from upstream
+
+    // ---- the rows of the stream --------------------------------------------------------------------------------
+    const int T = min(p.pr.keep_off[p.batch], p.part_rows);
+    if (p.have_draft) {
+        for (int b = warp; b < p.batch; b += AS_THREADS / 32) {
+            if (p.mode[b] != HS_ACCEPT_REJECTION) continue;
+            const int koff = p.pr.keep_off[b], nk = p.pr.n_keep[b];
+            for (int j = 1 + lane; j < nk; j += 32) {
+                const int par = p.pr.new_parent[koff + j];
+                const int k = koff + par;
+                if (par >= 0 && par < j && k < T) atomicOr(&s_bits[k >> 5], 1u << (k & 31));
+            }
+        }
+    }
+    // sequences that kept nothing (flagged upstream) and sequences in rejection mode without draft logits get their
+    // result here, shared out over the warps of the grid
+    for (int b = blockIdx.x * (AS_THREADS / 32) + warp; b < p.batch; b += gridDim.x * (AS_THREADS / 32)) {
+        const int st = p.pr.status[b];
+        const bool empty = p.pr.n_keep[b] <= 0 || st != 0;
+        const bool nodraft = !empty && p.mode[b] == HS_ACCEPT_REJECTION && !p.have_draft;
+        if (empty || nodraft) {
+            const int cap = p.out.path_cap;
+            for (int j = lane; j < cap; j += 32) {
+                p.out.path_nodes[b * cap + j] = -1;
+                p.out.path_compact[b * cap + j] = -1;
+                p.out.path_tokens[b * cap + j] = -1;
+            }
+            if (lane == 0) {
+                p.out.accept_len[b] = 0; p.out.bonus_token[b] = -1; p.out.terminal_rank[b] = -1;
+                p.out.status[b] = empty ? (st != 0 ? st : HS_ERR_BAD_TREE) : HS_ERR_INVALID_ARG;
+            }
+        }
+    }
+    __syncthreads();
+    if (warp == 0) {
+        constexpr int WPL = NWORDS / 32;
+        int c = 0;
+#pragma unroll
+        for (int i = 0; i < WPL; ++i) c += __popc(s_bits[lane * WPL + i]);
+        int incl = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int up = __shfl_up_sync(HS_FULL_MASK, incl, o);
+            if (lane >= o) incl += up;
+        }
+        int run = incl - c;
+#pragma unroll
+        for (int i = 0; i < WPL; ++i) {
+            s_pref[lane * WPL + i] = run;
+            run += __popc(s_bits[lane * WPL + i]);
+        }
+        if (lane == 31) s_pref[NWORDS] = run;
+    }
+    __syncthreads();
+    const int W = T + s_pref[NWORDS];
+    const long long total = (long long)W * p.nvec;
+    long long per = (total + gridDim.x - 1) / gridDim.x;
+    per = max(per, (long long)((p.nvec + (AS_MAX_SEGS - 2) - 1) / (AS_MAX_SEGS - 2)));   // a row in at most AS_MAX_SEGS shares
+    per = max(per, (long long)AS_ITEM_VECS);
+    const long long g0 = (long long)blockIdx.x * per, g1 = min(g0 + per, total);
+    if (g0 >= g1) return;
+    const int w_first = (int)(g0 / p.nvec), w_last = (int)((g1 - 1) / p.nvec);
+
+    auto lookup = [&](int w) -> WorkRow {
+        WorkRow r;
+        if (w < T) {
+            r.k = w; r.which = 0;
+        } else {
+            const int rnk = w - T;                        // the rnk-th set bit
+            int lo = 0, hi = NWORDS;
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (s_pref[mid] <= rnk) lo = mid; else hi = mid;
+            }
+            r.k = lo * 32 + (int)__fns(s_bits[lo], 0, rnk - s_pref[lo] + 1);
+            r.which = 1;
+        }
+        int lo = 0, hi = p.batch;                         // the last b with keep_off[b] <= k (skips empty sequences)
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (p.pr.keep_off[mid] <= r.k) lo = mid; else hi = mid;
+        }
+        r.b = lo;
+        r.nk = p.pr.n_keep[lo];
+        r.mode = p.mode[lo];
+        r.invT = LOG2E / p.temperature[lo];
+        const int orig_row = p.node_off[lo] + p.pr.keep_idx[r.k];
+        const int row = r.which == 1 ? orig_row : (p.target_layout == HS_ROWS_ORIGINAL ? orig_row : r.k);
+        r.ptr = (const char*)(r.which == 1 ? p.draft : p.target) + (size_t)row * p.row_stride * esz;
+        return r;
+    };
+
+    if (warp == AS_NW) {
+        // ---- producer warp: lane 0 walks the share item by item; all lanes look rows up, 32 rows at a time ---------
+        long long g = g0;
+        int it = 0, slot = 0;
+        unsigned int epar = 1u;              // parity of the slot's `empty` barrier before its first completion
+        for (int w = w_first; w <= w_last; ++w) {
+            const int rl = w - w_first;
+            if ((rl & 31) == 0) {
+                // (the consumers are at most AS_SLOTS + 1 rows behind: the other half of the ring)
+                if (w + lane <= w_last) s_rows[(rl + lane) % AS_ROW_RING] = lookup(w + lane);
+                __syncwarp();
+            }
+            if (lane == 0) {
+                const char* ptr = s_rows[rl % AS_ROW_RING].ptr;
+                const long long row_g0 = (long long)w * p.nvec;
+                int v = (int)(g - row_g0);
+                const int v_end = (int)(min(g1, row_g0 + p.nvec) - row_g0);
+                while (v < v_end) {
+                    const int len = min(AS_ITEM_VECS, v_end - v);
+                    if (it >= AS_SLOTS) mbar_wait(smem_u32(&s_empty[slot]), epar, p.err);
+                    const unsigned int bar = smem_u32(&s_full[slot]);
+                    // (the arrival below also publishes the row table to the consumers that wait on this barrier)
+                    mbar_expect_tx(bar, (unsigned int)len * 16u);
+                    bulk_load(slots0 + (unsigned int)slot * (AS_ITEM_VECS * 16), ptr + (size_t)v * 16, (unsigned int)len * 16u, bar);
+                    v += len;
+                    ++it;
+                    if (++slot == AS_SLOTS) { slot = 0; epar ^= 1u; }
+                }
+                g = row_g0 + v_end;
+            }
+            __syncwarp();
+        }
+        return;
+    }
+
+    // ---- consumers -------------------------------------------------------------------------------------------------
+    const unsigned int ninf = BF16 ? 0xff80ff80u : 0xff800000u;
+    int cslot = 0;                 // slot of the next item and the parity of its `full` barrier (the producer fills
+    unsigned int cpar = 0u;        // the slots round-robin in the same order)
+    int seg = 0;
+    long long g = g0;
+    while (g < g1) {
+        // ---- one segment: the part of this share inside row w of the stream --------------------------------------
+        const int w = (int)(g / p.nvec);
+        const long long row_g0 = (long long)w * p.nvec;
+        const int sv0 = (int)(g - row_g0);
+        const int sv1 = (int)(min(g1, row_g0 + p.nvec) - row_g0);
+        mbar_wait(smem_u32(&s_full[cslot]), cpar, p.err);      // the row's first item; the row table entry with it
+        const WorkRow r = s_rows[(w - w_first) % AS_ROW_RING];
+        const bool sampling = r.mode != HS_ACCEPT_GREEDY;      // the row's normaliser is needed
+        const bool want_arg = r.which == 0;
+        unsigned int bm = ninf, bc = 0u;      // bf16: running maximum and position code of the two half-lanes
+        float m_f = -CUDART_INF_F;            // f32: running maximum and its position code
+        unsigned int c_f = 0u;
+        float m_t = -CUDART_INF_F;            // maximum the sums are relative to
+        float2 s2 = make_float2(0.f, 0.f);
+        int it = 0;
+        for (int v = sv0; v < sv1; ++it) {
+            const int len = min(AS_ITEM_VECS, sv1 - v);
+            const int slot = cslot;
+            mbar_wait(smem_u32(&s_full[slot]), cpar, p.err);
+            if (++cslot == AS_SLOTS) { cslot = 0; cpar ^= 1u; }
+            const uint4* st = reinterpret_cast<const uint4*>(slots_gen + (size_t)slot * (AS_ITEM_VECS * 16));
+            uint4 d[AS_VPT];
+            if (len == AS_ITEM_VECS) {
+#pragma unroll
+                for (int j = 0; j < AS_VPT; ++j) d[j] = st[tid + j * AS_CONSUMERS];
+            } else {
+#pragma unroll
+                for (int j = 0; j < AS_VPT; ++j) {
+                    const int vl = tid + j * AS_CONSUMERS;
+                    d[j] = (vl < len) ? st[vl] : make_uint4(ninf, ninf, ninf, ninf);
+                }
+            }
+            if (v + len == p.nvec && p.nvec * VE != p.vocab) {                // the row's last vector runs past vocab
+#pragma unroll
+                for (int j = 0; j < AS_VPT; ++j) {
+                    if (v + tid + j * AS_CONSUMERS == p.nvec - 1) {
+                        unsigned int* wd = reinterpret_cast<unsigned int*>(&d[j]);
+#pragma unroll
+                        for (int e = 0; e < VE; ++e)
+                            if ((p.nvec - 1) * VE + e >= p.vocab) {
+                                if (BF16) wd[e >> 1] = (e & 1) ? ((wd[e >> 1] & 0x0000ffffu) | 0xff800000u)
+                                                               : ((wd[e >> 1] & 0xffff0000u) | 0x0000ff80u);
+                                else wd[e] = 0xff800000u;
+                            }
+                    }
+                }
+            }
+            // maxima (target rows: with the position of the first occurrence; items, vectors and words are taken in
+            // ascending token order and only a strictly larger value replaces the running one)
+            if (BF16) {
+#pragma unroll
+                for (int j = 0; j < AS_VPT; ++j) {
+                    const unsigned int* wd = reinterpret_cast<const unsigned int*>(&d[j]);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const __nv_bfloat162 x2 = *reinterpret_cast<const __nv_bfloat162*>(&wd[q]);
+                        const __nv_bfloat162 m2 = *reinterpret_cast<const __nv_bfloat162*>(&bm);
+                        if (want_arg) {
+                            const unsigned int gt = __hgt2_mask(x2, m2);
+                            const unsigned int cc = ((unsigned int)(it << 4 | j << 2 | q)) * 0x00010001u;
+                            bc = (bc & ~gt) | (cc & gt);
+                        }
+                        const __nv_bfloat162 n2 = __hmax2(m2, x2);
+                        bm = *reinterpret_cast<const unsigned int*>(&n2);
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < AS_VPT; ++j) {
+                    const unsigned int* wd = reinterpret_cast<const unsigned int*>(&d[j]);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float x = __uint_as_float(wd[e]);
+                        if (x > m_f) { m_f = x; c_f = (unsigned int)(it << 4 | j << 2 | e); }
+                    }
+                }
+            }
+            if (sampling) {
+                const float imax = BF16 ? fmaxf(bf16_lo(bm), bf16_hi(bm)) : m_f;
+                if (imax > m_t) {                     // the thread's maximum grows: rescale its sum
+                    const float f = (m_t == -CUDART_INF_F) ? 0.f : ex2a((m_t - imax) * r.invT);
+                    s2.x *= f; s2.y *= f;
+                    m_t = imax;
+                }
+                const float nml = (m_t == -CUDART_INF_F) ? 0.f : -m_t * r.invT;
+                const float2 l2 = make_float2(r.invT, r.invT), n2 = make_float2(nml, nml);
+                const unsigned int floor2 = 0xf149f149u;  // bf16 pair of -1e30: keeps 0 * x finite for x = -inf
+#pragma unroll
+                for (int j = 0; j < AS_VPT; ++j) {
+                    const unsigned int* wd = reinterpret_cast<const unsigned int*>(&d[j]);
+                    if (BF16) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const __nv_bfloat162 cl = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&wd[q]),
+                                                             *reinterpret_cast<const __nv_bfloat162*>(&floor2));
+                            const unsigned int cw = *reinterpret_cast<const unsigned int*>(&cl);
+                            const float2 t = fma2_ftz(make_float2(bf16_lo(cw), bf16_hi(cw)), l2, n2);
+                            s2 = add2_ftz(s2, make_float2(ex2a(t.x), ex2a(t.y)));
+                        }
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 2; ++q) {
+                            const float2 x = make_float2(fmaxf(__uint_as_float(wd[2 * q]), -1e30f),
+                                                         fmaxf(__uint_as_float(wd[2 * q + 1]), -1e30f));
+                            const float2 t = fma2_ftz(x, l2, n2);
+                            s2 = add2_ftz(s2, make_float2(ex2a(t.x), ex2a(t.y)));
+                        }
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));
+            v += len;
+        }
+        // ---- end of the segment: the thread's candidates become (value, lowest index) keys ------------------------
+        unsigned long long key = 0ull;
+        if (want_arg) {
+            if (BF16) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const float val = h ? bf16_hi(bm) : bf16_lo(bm);
+                    const unsigned int code = (bc >> (16 * h)) & 0xffffu;
+                    if (val > -CUDART_INF_F) {
+                        const int vec = sv0 + (int)(code >> 4) * AS_ITEM_VECS + tid + (int)((code >> 2) & 3u) * AS_CONSUMERS;
+                        const unsigned long long kk = make_key(val, vec * 8 + 2 * (int)(code & 3u) + h);
+                        key = kk > key ? kk : key;
+                    }
+                }
+            } else if (m_f > -CUDART_INF_F) {
+                const int vec = sv0 + (int)(c_f >> 4) * AS_ITEM_VECS + tid + (int)((c_f >> 2) & 3u) * AS_CONSUMERS;
+                key = make_key(m_f, vec * 4 + (int)(c_f & 3u));
+            }
+            key = warp_max_u64(key);
+        }
+        float wm = -CUDART_INF_F, ws = 0.f;
+        if (sampling) {
+            wm = warp_max(m_t);
+            const float f = (m_t == -CUDART_INF_F) ? 0.f : ex2a((m_t - wm) * r.invT);
+            ws = warp_sum((s2.x + s2.y) * f);
+        }
+        if (lane == 0) { s_wkey[seg & 1][warp] = key; s_wms[seg & 1][warp] = make_float2(wm, ws); }
+        named_bar_sync(1, AS_CONSUMERS);
+        if (warp == 0) {
+            // the other warps are already on their way to the next segment
+            unsigned long long best = warp_max_u64(lane < AS_NW ? s_wkey[seg & 1][lane] : 0ull);
+            const float2 ms = lane < AS_NW ? s_wms[seg & 1][lane] : make_float2(-CUDART_INF_F, 0.f);
+            float M = warp_max(ms.x);
+            float S = sampling ? warp_sum(ms.x == -CUDART_INF_F ? 0.f : ms.y * ex2a((ms.x - M) * r.invT)) : 0.f;
+            const int c_first = (int)(row_g0 / per);
+            const int nseg = (int)((row_g0 + p.nvec - 1) / per) - c_first + 1;
+            bool mine = true;                     // this warp holds the row's final result
+            if (nseg > 1) {
+                // a share holds at most two partial rows: the one that began in an earlier share, the one that goes on
+                auto slot_of = [&](int c) { return 2 * c + (row_g0 < (long long)c * per ? 0 : 1); };
+                int last = 0;
+                if (lane == 0) {
+                    p.partials[slot_of(blockIdx.x)] =
+                        make_uint4((unsigned int)best, (unsigned int)(best >> 32), __float_as_uint(M), __float_as_uint(S));
+                    // one release-acquire arrival at device scope: the partial is visible to whoever arrives last
+                    int old;
+                    asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(old) : "l"(&p.row_cnt[w]) : "memory");
+                    last = old == nseg - 1;
+                    if (last) p.row_cnt[w] = 0;
+                }
+                mine = __shfl_sync(HS_FULL_MASK, last, 0) != 0;
+                if (mine) {
+                    unsigned long long ck = 0ull;
+                    float cm = -CUDART_INF_F, cs = 0.f;
+                    if (lane < nseg) {
+                        const uint4 q = __ldcg(&p.partials[slot_of(c_first + lane)]);
+                        ck = ((unsigned long long)q.y << 32) | q.x;
+                        cm = __uint_as_float(q.z);
+                        cs = __uint_as_float(q.w);
+                    }
+                    best = warp_max_u64(ck);
+                    M = warp_max(cm);
+                    S = sampling ? warp_sum(cm == -CUDART_INF_F ? 0.f : cs * ex2a((cm - M) * r.invT)) : 0.f;
+                }
+            }
+            if (mine && lane == 0) {
+                if (r.which == 0) {
+                    p.ro.tgt_arg[r.k] = key_index(best);
+                    p.ro.tgt_ms[r.k] = make_float2(M, S);
+                    if (r.mode != HS_ACCEPT_REJECTION) {
+                        // greedy sequences and deterministic proposals finish in this kernel: the CTA that completes a
+                        // sequence's last target row walks its tree once its own share is done
+                        int old;
+                        asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(old) : "l"(&p.seq_cnt[r.b]) : "memory");
+                        if (old == r.nk - 1) {
+                            p.seq_cnt[r.b] = 0;
+                            s_pending[s_npending++] = (unsigned short)r.b;
+                        }
+                    }
+                } else {
+                    p.ro.drf_ms[r.k] = make_float2(M, S);
+                }
+            }
+        }
+        ++seg;
+        g = row_g0 + sv1;
+    }
+    named_bar_sync(1, AS_CONSUMERS);          // warp 0 has finished its last row: the list of walks is complete
+    if (tid < HS_ROW_THREADS) {
+        const int npend = s_npending;
+        for (int i = 0; i < npend; ++i) {
+            const int b = s_pending[i];
+            if (p.mode[b] == HS_ACCEPT_GREEDY) greedy_walk(p, b);
+            else deterministic_walk(p, b);
+            walk_sync();                       // the walks' shared arrays are free again
+        }
     }
 }
 
@@ -861,17 +1278,34 @@ hs_status hs_launch_accept(hs_ctx* ctx, const hs_tree_batch* tree, const hs_prun
     p.ro.drf_ms = (float2*)(ctx->scratch + o); o += hs_align_up((size_t)rows * sizeof(float2), 256);
     p.partials = (uint4*)(ctx->scratch + o);
     p.part_rows = rows;
-    o += (size_t)2 * rows * p.chunks * sizeof(uint4);
+    // (chunk kernel: a partial per chunk of a row; streaming kernel: two per share, one share per SM)
+    o += max((size_t)2 * rows * p.chunks, (size_t)2 * ctx->sm_count) * sizeof(uint4);
     if (o > ctx->scratch_bytes) return HS_ERR_WORKSPACE;
     p.row_cnt = ctx->counters + HS_CNT_ACC_ROW;
     p.seq_cnt = ctx->counters + HS_CNT_ACC_SEQ;
     p.err = ctx->counters + HS_CNT_ERROR;
     p.staged = 0;
     // without draft logits every sequence must be greedy: no draft rows to scan and no sampling walk
-    dim3 grid(p.chunks, rows, p.have_draft ? 2 : 1);
-    cudaError_t e = dtype == HS_BF16
-        ? hs_launch(accept_rows_kernel<true>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p)
-        : hs_launch(accept_rows_kernel<false>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p);
+    cudaError_t e;
+    const bool streamed = ctx->row_pass == HS_ROW_PASS_STREAM ||
+                          (ctx->row_pass == HS_ROW_PASS_AUTO && (size_t)rows * p.nvec * 16 >= AS_MIN_BYTES);
+    if (streamed) {
+        // enough rows to be bound by memory traffic: one persistent CTA per SM streams them
+        if (!ctx->rows_ready) {
+            if (cudaFuncSetAttribute(accept_stream_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AS_SMEM_BYTES) != cudaSuccess ||
+                cudaFuncSetAttribute(accept_stream_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, AS_SMEM_BYTES) != cudaSuccess)
+                return HS_ERR_CUDA;
+            ctx->rows_ready = true;
+        }
+        e = dtype == HS_BF16
+            ? hs_launch(accept_stream_kernel<true>, dim3(ctx->sm_count), dim3(AS_THREADS), AS_SMEM_BYTES, stream, ctx->pdl, dim3(1, 1, 1), p)
+            : hs_launch(accept_stream_kernel<false>, dim3(ctx->sm_count), dim3(AS_THREADS), AS_SMEM_BYTES, stream, ctx->pdl, dim3(1, 1, 1), p);
+    } else {
+        dim3 grid(p.chunks, rows, p.have_draft ? 2 : 1);
+        e = dtype == HS_BF16
+            ? hs_launch(accept_rows_kernel<true>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p)
+            : hs_launch(accept_rows_kernel<false>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p);
+    }
     if (e != cudaSuccess) return HS_ERR_CUDA;
     if (!p.have_draft) return HS_OK;
     // the cluster shape of the walk is fixed at compile time (__cluster_dims__); its two row slices in shared memory

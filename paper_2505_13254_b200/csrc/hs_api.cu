@@ -70,9 +70,11 @@ extern "C" hs_status hs_create(hs_ctx** out, int32_t device, size_t workspace_by
     const char* no_pdl = getenv("HS_DISABLE_PDL");
     c->pdl = !(no_pdl && no_pdl[0] == '1');
     c->prefetch = 0;
+    c->row_pass = HS_ROW_PASS_AUTO;
     c->attn_ready = false;
     c->walk_ready = false;
     c->quant_ready = false;
+    c->rows_ready = false;
     if (cudaDeviceSynchronize() != cudaSuccess) { cudaFree(p); delete c; return HS_ERR_CUDA; }
     *out = c;
     return HS_OK;
@@ -104,6 +106,12 @@ hs_status hs_launch_wait_selftest(hs_ctx* ctx, uint64_t limit_ns, cudaStream_t s
 extern "C" hs_status hs_set_prefetch(hs_ctx* ctx, int32_t flags) {
     if (!ctx || (flags & ~(HS_PREFETCH_LOGITS | HS_PREFETCH_KV))) return HS_ERR_INVALID_ARG;
     ctx->prefetch = flags;
+    return HS_OK;
+}
+
+extern "C" hs_status hs_set_row_pass(hs_ctx* ctx, int32_t variant) {
+    if (!ctx || variant < HS_ROW_PASS_AUTO || variant > HS_ROW_PASS_STREAM) return HS_ERR_INVALID_ARG;
+    ctx->row_pass = variant;
     return HS_OK;
 }
 

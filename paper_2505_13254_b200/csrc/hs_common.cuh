@@ -25,10 +25,12 @@ struct hs_ctx {
     size_t scratch_bytes;
     void* encode_tiled; // cuTensorMapEncodeTiled entry point
     bool pdl;           // launch kernels with programmatic stream serialisation
+    int row_pass;       // HS_ROW_PASS_*: kernel of the acceptance row pass
     int prefetch;       // HS_PREFETCH_* bits: inputs a kernel may fetch before its dependency wait
     bool attn_ready;    // attention kernel attributes set and cluster capacities queried on this device
     int attn_cap[9];    // CTAs of the attention kernel that run at once in clusters of s = 1..8
     bool walk_ready;    // acceptance walk kernel attributes set on this device
+    bool rows_ready;    // streaming acceptance row pass: shared-memory attribute set on this device
     bool quant_ready;   // streaming entropy kernel: shared-memory attribute set on this device
 };
 

@@ -65,6 +65,10 @@ __device__ __forceinline__ void bulk_load(unsigned int dst, const void* src, uns
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
+// Barrier `id` (1..15; 0 is __syncthreads' own) over `nthr` threads of the CTA (a multiple of 32).
+__device__ __forceinline__ void named_bar_sync(int id, int nthr) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthr) : "memory");
+}
 __device__ __forceinline__ void tma_load_3d(unsigned int dst, const CUtensorMap* tm, int c0, int c1, int c2,
                                             unsigned int bar) {
     asm volatile(
