@@ -353,7 +353,12 @@ def main():
     quant_bytes = n_rows * cfg.vocab * esz
     L = int(np.diff(batch["kv_off"]).sum())
     attn_bytes = 2 * (L + nk) * cfg.hkv * cfg.head_dim * 2 + 2 * nk * cfg.hq * cfg.head_dim * 2
-    accept_bytes = nk * cfg.vocab * esz
+    # rows the acceptance reads: the target row of every kept node and, in rejection mode, the draft row of every kept
+    # node that has a kept child
+    koff, npar, modes = st.pruned.keep_off.cpu().numpy(), st.pruned.new_parent.cpu().numpy(), db0.mode.cpu().numpy()
+    draft_rows = sum(len(set(int(x) for x in npar[koff[b]:koff[b + 1]] if x >= 0))
+                     for b in range(cfg.batch) if modes[b] == hb.HS_ACCEPT_REJECTION and db0.any_sampling)
+    accept_bytes = (nk + draft_rows) * cfg.vocab * esz
     kern = {
         "quantify": {"bytes": quant_bytes, "us": call_us["quantify"], "launches_per_step": 2},
         "attention": {"bytes": attn_bytes, "us": call_us["attention"], "launches_per_step": 1},

@@ -1060,7 +1060,6 @@ accept_walk_kernel(const AcceptParams p) {
     __shared__ unsigned long long s_x[2][WALK_CLUSTER];    // all-gather buffers of the cluster exchanges
     unsigned int xch = 0;                  // exchanges through s_cta so far
     __shared__ int s_pick[2];
-    __shared__ int s_child;
     const int tid = threadIdx.x;
     const int b = blockIdx.x / WALK_CLUSTER;
     const unsigned int rank = cluster.block_rank();
