@@ -228,6 +228,15 @@ hs_status hs_entropy_quantify_static(const hs_tree_batch* tree, const void* draf
                                      int64_t row_stride, int32_t vocab, const hs_policy* policy,
                                      const hs_quant_out* out, hs_stream stream);
 
+/* hs_entropy_quantify and hs_stratify_prune (Sec. 4.1 - 4.3, reranking of Sec. 2.2) as one call of two launches
+ * instead of three: the kernel that computes the tree scores of a sequence goes on to prune it, from shared memory
+ * and registers.  Arguments, outputs (all of `quant` and all of `pruned` are written) and error behaviour are those
+ * of the two calls made one after the other; the budgeted variant has no fused form.  Device pointers; enqueues on
+ * `stream` and returns. */
+hs_status hs_entropy_quantify_prune(hs_ctx* ctx, const hs_tree_batch* tree, const void* draft_logits,
+                                    hs_dtype dtype, int64_t row_stride, int32_t vocab, const hs_policy* policy,
+                                    const hs_quant_out* quant, const hs_pruned_tree* pruned, hs_stream stream);
+
 /* Sec. 4.2-4.3 and the reranking of Sec. 2.2.  Reads score, phi_star, depth, status of `quant`. */
 hs_status hs_stratify_prune(hs_ctx* ctx, const hs_tree_batch* tree, const hs_quant_out* quant,
                             const hs_policy* policy, const hs_pruned_tree* out, hs_stream stream);

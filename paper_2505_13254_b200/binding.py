@@ -69,7 +69,7 @@ class _AcceptOut(C.Structure):
 
 EXPORTS = ("hs_status_string", "hs_workspace_bytes", "hs_create", "hs_destroy", "hs_device_error", "hs_entropy_quantify",
            "hs_stratify_prune", "hs_tree_verify_attention", "hs_accept_path", "hs_philox_uniforms",
-           "hs_entropy_quantify_static", "hs_set_prefetch", "hs_set_row_pass", "hs_selftest_wait_timeout", "hs_expand_init",
+           "hs_entropy_quantify_static", "hs_set_prefetch", "hs_set_row_pass", "hs_entropy_quantify_prune", "hs_selftest_wait_timeout", "hs_expand_init",
            "hs_expand_level", "hs_rerank", "hs_cart_fit", "hs_cart_workspace_bytes", "hs_stratify_prune_budget")
 
 
@@ -92,6 +92,8 @@ def lib() -> C.CDLL:
         L.hs_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_uint64, vp]
         L.hs_entropy_quantify.argtypes = [C.c_void_p, C.POINTER(_TreeBatch), vp, C.c_int, C.c_int64, C.c_int32,
                                           C.POINTER(_Policy), C.POINTER(_QuantOut), vp]
+        L.hs_entropy_quantify_prune.argtypes = [C.c_void_p, C.POINTER(_TreeBatch), vp, C.c_int, C.c_int64, C.c_int32,
+                                                C.POINTER(_Policy), C.POINTER(_QuantOut), C.POINTER(_PrunedTree), vp]
         L.hs_entropy_quantify_static.argtypes = [C.POINTER(_TreeBatch), vp, C.c_int, C.c_int64, C.c_int32,
                                                  C.POINTER(_Policy), C.POINTER(_QuantOut), vp]
         L.hs_stratify_prune.argtypes = [C.c_void_p, C.POINTER(_TreeBatch), C.POINTER(_QuantOut),
@@ -289,6 +291,20 @@ def hs_entropy_quantify_static(tree: TreeBatch, draft_logits: torch.Tensor, poli
                                             draft_logits.stride(0), draft_logits.shape[1], C.byref(p), C.byref(o),
                                             _stream()), "hs_entropy_quantify_static")
     return out
+
+
+def hs_entropy_quantify_prune(ctx: Context, tree: TreeBatch, draft_logits: torch.Tensor, policy: dict,
+                              out: Optional[QuantOut] = None, pruned_out: Optional["PrunedTree"] = None):
+    """hs_entropy_quantify followed by hs_stratify_prune, as one call of two launches."""
+    if out is None:
+        out = QuantOut(tree.n_nodes_total, tree.batch, policy["top_k"], draft_logits.device)
+    if pruned_out is None:
+        pruned_out = PrunedTree(tree.n_nodes_total, tree.batch, tree.parent.device)
+    t, p, o, q = tree.c(), make_policy(policy), out.c(), pruned_out.c()
+    _check(lib().hs_entropy_quantify_prune(ctx.handle, C.byref(t), _ptr(draft_logits), _dtype_code(draft_logits),
+                                           draft_logits.stride(0), draft_logits.shape[1], C.byref(p), C.byref(o),
+                                           C.byref(q), _stream()), "hs_entropy_quantify_prune")
+    return out, pruned_out
 
 
 def hs_stratify_prune(ctx: Context, tree: TreeBatch, quant: QuantOut, policy: dict,

@@ -166,6 +166,29 @@ extern "C" hs_status hs_entropy_quantify(hs_ctx* ctx, const hs_tree_batch* tree,
     return hs_launch_quantify(ctx, tree, draft_logits, dtype, row_stride, vocab, policy, out, (cudaStream_t)stream);
 }
 
+static bool pruned_out_ok(const hs_pruned_tree* out) {
+    return out && out->bin && out->d_prime && out->n_prime && out->n_keep && out->keep_off && out->keep_idx &&
+           out->new_parent && out->new_depth && out->keep_rank && out->anc_mask && out->status;
+}
+
+extern "C" hs_status hs_entropy_quantify_prune(hs_ctx* ctx, const hs_tree_batch* tree, const void* draft_logits,
+                                               hs_dtype dtype, int64_t row_stride, int32_t vocab,
+                                               const hs_policy* policy, const hs_quant_out* quant,
+                                               const hs_pruned_tree* pruned, hs_stream stream) {
+    if (!ctx || !quant || !hs_on_device(ctx)) return HS_ERR_INVALID_ARG;
+    if (!tree_ok(tree) || !policy_ok(policy) || !logits_ok(draft_logits, dtype, row_stride, vocab))
+        return HS_ERR_INVALID_ARG;
+    if (!quant->row_max || !quant->row_lse || !quant->h_full || !quant->i_topk || !quant->i_trunc || !quant->topk_val ||
+        !quant->topk_idx || !quant->logc || !quant->score || !quant->phi || !quant->depth || !quant->pstar_node ||
+        !quant->phi_star || !quant->status || !pruned_out_ok(pruned))
+        return HS_ERR_INVALID_ARG;
+    hs_status st = hs_launch_quantify(ctx, tree, draft_logits, dtype, row_stride, vocab, policy, quant,
+                                      (cudaStream_t)stream, false);
+    if (st != HS_OK) return st;
+    return hs_launch_tree_prune(ctx, tree, draft_logits, dtype, row_stride, vocab, policy, quant, pruned,
+                                (cudaStream_t)stream);
+}
+
 extern "C" hs_status hs_stratify_prune(hs_ctx* ctx, const hs_tree_batch* tree, const hs_quant_out* quant,
                                        const hs_policy* policy, const hs_pruned_tree* out, hs_stream stream) {
     if (!ctx || !quant || !out || !hs_on_device(ctx)) return HS_ERR_INVALID_ARG;

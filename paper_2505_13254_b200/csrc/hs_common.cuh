@@ -157,7 +157,10 @@ __device__ __forceinline__ float philox_uniform(unsigned long long seed, unsigne
 // ---- launchers implemented in the kernel files ---------------------------------------------
 hs_status hs_launch_quantify(hs_ctx* ctx, const hs_tree_batch* tree, const void* logits, hs_dtype dtype,
                              int64_t row_stride, int32_t vocab, const hs_policy* policy,
-                             const hs_quant_out* out, cudaStream_t stream);
+                             const hs_quant_out* out, cudaStream_t stream, bool with_tree_stage = true);
+hs_status hs_launch_tree_prune(hs_ctx* ctx, const hs_tree_batch* tree, const void* logits, hs_dtype dtype,
+                               int64_t row_stride, int32_t vocab, const hs_policy* policy, const hs_quant_out* quant,
+                               const hs_pruned_tree* out, cudaStream_t stream);
 hs_status hs_launch_stratify_prune(hs_ctx* ctx, const hs_tree_batch* tree, const hs_quant_out* quant,
                                    const hs_policy* policy, const hs_pruned_tree* out, cudaStream_t stream);
 hs_status hs_launch_stratify_prune_budget(hs_ctx* ctx, const hs_tree_batch* tree, const hs_quant_out* quant,

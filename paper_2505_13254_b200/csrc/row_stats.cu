@@ -23,6 +23,7 @@
 #include "hs_common.cuh"
 #include "hs_layout.h"
 #include "hs_ptx.cuh"
+#include "tree_stage.cuh"
 
 #define CAND_CAP 512
 #define LOG2E 1.4426950408889634f
@@ -584,89 +585,9 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
 // Tree stage: one CTA of 128 threads per sequence, one thread per node
 // ================================================================================================================
 __global__ void __launch_bounds__(HS_MAX_NODES) tree_scores_kernel(const QuantParams p) {
-    __shared__ float s_logc[HS_MAX_NODES], s_I[HS_MAX_NODES], s_phi[HS_MAX_NODES];
-    __shared__ int s_par[HS_MAX_NODES];
-    __shared__ unsigned long long s_best[4];
-    __shared__ int s_maxd[4];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int b = blockIdx.x;
+    __shared__ TreeStageSmem sm;
     pdl_launch_dependents();
-    // The tree and the logit of every node's token are inputs of the call, not results of the row pass: if the caller
-    // vouches that they were complete before the call (prefetch), they are fetched while the row pass still runs.
-    if (!p.prefetch) pdl_wait();
-    const int base = p.node_off[b];
-    const int n = p.node_off[b + 1] - base;
-    // validation
-    int bad = (n > HS_MAX_NODES || n <= 0);
-    int par = -1, tok = 0;
-    if (!bad && tid < n) {
-        par = p.parent[base + tid];
-        tok = p.token[base + tid];
-        if (tid == 0) bad = (par != -1);
-        else bad = (par < 0 || par >= tid || tok < 0 || tok >= p.vocab);
-    }
-    float lv = 0.f;
-    if (!bad && tid < n && tid > 0) {
-        const size_t off = (size_t)(base + par) * p.row_stride + tok;
-        lv = p.is_bf16 ? __bfloat162float(((const __nv_bfloat16*)p.logits)[off]) : ((const float*)p.logits)[off];
-    }
-    if (p.prefetch) pdl_wait();                   // the row statistics come from the kernel ahead
-    bad = __syncthreads_or(bad);
-    if (bad) {
-        for (int i = tid; i < n; i += blockDim.x) {
-            p.out.logc[base + i] = 0.f; p.out.score[base + i] = 0.f; p.out.phi[base + i] = 0.f;
-            p.out.depth[base + i] = 0;
-        }
-        if (tid == 0) { p.out.status[b] = HS_ERR_BAD_TREE; p.out.pstar_node[b] = 0; p.out.phi_star[b] = 0.f; }
-        return;
-    }
-    if (tid < n) {
-        float lc = 0.f;
-        if (tid > 0) lc = lv - p.out.row_lse[base + par];
-        s_logc[tid] = lc;
-        s_I[tid] = p.entropy_mode == 0 ? p.out.i_topk[base + tid] : p.out.i_trunc[base + tid];
-        s_par[tid] = par;
-    }
-    __syncthreads();
-    float S = 0.f, Phi = 0.f;
-    int dep = 0;
-    if (tid < n) {
-        int a = tid;
-        while (a > 0) {
-            const int pa = s_par[a];
-            S += s_logc[a];
-            Phi += s_I[pa];
-            a = pa;
-            ++dep;
-        }
-        if (p.phi_mode == 1) Phi += s_I[tid];
-        s_phi[tid] = Phi;
-        p.out.logc[base + tid] = s_logc[tid];
-        p.out.score[base + tid] = S;
-        p.out.phi[base + tid] = Phi;
-        p.out.depth[base + tid] = dep;
-    }
-    // deepest level, then P* among the nodes of depth min(d_base, deepest)
-    int md = dep;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) md = max(md, __shfl_xor_sync(HS_FULL_MASK, md, o));
-    if (lane == 0) s_maxd[warp] = md;
-    __syncthreads();
-    md = max(max(s_maxd[0], s_maxd[1]), max(s_maxd[2], s_maxd[3]));
-    const int t_eval = min(p.d_base, md);
-    unsigned long long key = 0ull;
-    if (tid < n && dep == t_eval) key = make_key(p.pstar_mode == 0 ? s_logc[tid] : S, tid);
-    key = warp_max_u64(key);
-    if (lane == 0) s_best[warp] = key;
-    __syncthreads();
-    if (tid == 0) {
-        unsigned long long best = s_best[0];
-        for (int w = 1; w < 4; ++w) best = s_best[w] > best ? s_best[w] : best;
-        const int node = key_index(best);
-        p.out.pstar_node[b] = node;
-        p.out.phi_star[b] = s_phi[node];
-        p.out.status[b] = HS_OK;
-    }
+    tree_stage_cta(p, blockIdx.x, sm);
 }
 
 static void fill_common(QuantParams& p, const hs_tree_batch* tree, const void* logits, hs_dtype dtype,
@@ -737,7 +658,7 @@ static void quantify_geometry(int rows, int nvec, int sm_count, QuantParams& p, 
 
 hs_status hs_launch_quantify(hs_ctx* ctx, const hs_tree_batch* tree, const void* logits, hs_dtype dtype,
                              int64_t row_stride, int32_t vocab, const hs_policy* policy,
-                             const hs_quant_out* out, cudaStream_t stream) {
+                             const hs_quant_out* out, cudaStream_t stream, bool with_tree_stage) {
     QuantParams p;
     fill_common(p, tree, logits, dtype, row_stride, vocab, policy, out);
     if (p.nvec > QS_ITEM_VECS * 64) return HS_ERR_SHAPE;            // vocabulary beyond 2^20 bf16 / 2^19 fp32 logits
@@ -763,6 +684,7 @@ hs_status hs_launch_quantify(hs_ctx* ctx, const hs_tree_batch* tree, const void*
         ? hs_launch(quantify_stream_kernel<true>, dim3(nctas), dim3(QS_THREADS), smem, stream, ctx->pdl, dim3(1, 1, 1), p)
         : hs_launch(quantify_stream_kernel<false>, dim3(nctas), dim3(QS_THREADS), smem, stream, ctx->pdl, dim3(1, 1, 1), p);
     if (e != cudaSuccess) return HS_ERR_CUDA;
+    if (!with_tree_stage) return HS_OK;              // (the caller launches the kernel that also prunes)
     e = hs_launch(tree_scores_kernel, dim3(p.batch), dim3(HS_MAX_NODES), 0, stream, ctx->pdl, dim3(1, 1, 1), p);
     return e == cudaSuccess ? HS_OK : HS_ERR_CUDA;
 }

@@ -10,6 +10,7 @@
 #include "hs_common.cuh"
 #include "hs_layout.h"
 #include "hs_ptx.cuh"
+#include "tree_stage.cuh"
 
 struct PruneParams {
     int batch;
@@ -182,82 +183,72 @@ __global__ void __launch_bounds__(BUDGET_THREADS) budget_kernel(const PruneParam
     }
 }
 
-__global__ void __launch_bounds__(HS_MAX_NODES) stratify_prune_kernel(const PruneParams p) {
-    __shared__ float s_S[HS_MAX_NODES];
-    __shared__ int s_elig[HS_MAX_NODES];
-    __shared__ int s_new[HS_MAX_NODES];
-    __shared__ int s_par[HS_MAX_NODES];
-    __shared__ int s_warp[4];
-    __shared__ int s_off;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int b = blockIdx.x;
-    pdl_launch_dependents();
-    pdl_wait();                            // scores and Phi(P*) come from the kernel ahead in the stream
-    const int base = p.node_off[b];
-    const int n = min(p.node_off[b + 1] - base, HS_MAX_NODES);
+struct PruneSmem {
+    __align__(16) float S[HS_MAX_NODES];
+    int nw[HS_MAX_NODES], par[HS_MAX_NODES];
+    int warp[4];
+    int off;
+};
 
-    // offset of this sequence in the compacted arrays
-    int part = 0;
-    if (p.counted) {
-        for (int bb = tid; bb < b; bb += HS_MAX_NODES) part += p.out.n_keep[bb];
-    } else {
-        for (int bb = tid; bb < b; bb += HS_MAX_NODES) part += kept_count(p, bb);
-    }
+// Sum of `part` over the CTA's 128 threads, the same value in every thread.
+__device__ __forceinline__ int cta_sum(int part, PruneSmem& sm) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(HS_FULL_MASK, part, o);
-    if (lane == 0) s_warp[warp] = part;
+    __syncthreads();                       // sm.warp may still be read
+    if (lane == 0) sm.warp[warp] = part;
     __syncthreads();
-    if (tid == 0) s_off = s_warp[0] + s_warp[1] + s_warp[2] + s_warp[3];
-    __syncthreads();
-    const int off = s_off;
+    return sm.warp[0] + sm.warp[1] + sm.warp[2] + sm.warp[3];
+}
 
-    const int status = p.qstatus[b];
+// Reranking and compaction of sequence b by its CTA (thread t = node t with depth `dep`, parent `par`, ln V `S`):
+// Top-N' among the nodes of depth <= d' by (S descending, index ascending), ballot + prefix compaction, parents
+// re-indexed, ancestor-or-self masks.  `offset_of(n_keep)` returns where the sequence starts in the compacted arrays.
+template <class OffsetFn>
+__device__ __forceinline__ void prune_cta(const PruneParams& p, int b, int n, int status, float phi_star, int dep,
+                                          int par, float S, PruneSmem& sm, OffsetFn offset_of) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int bin = 0, dp = 0, np = 0;
-    policy_lookup(p, p.phi_star[b], bin, dp, np);
-
-    int dep = 0, par = -1;
-    float S = 0.f;
-    bool elig = false;
-    if (tid < n && status == 0) {
-        dep = p.depth[base + tid];
-        par = p.parent[base + tid];
-        S = p.score[base + tid];
-        elig = dep <= dp;
-    }
-    s_S[tid] = S;
-    s_elig[tid] = elig;
-    s_par[tid] = par;
+    policy_lookup(p, phi_star, bin, dp, np);
+    const bool elig = tid < n && status == 0 && dep <= dp;
+    // rank among eligible nodes by (S descending, index ascending): a node that is not eligible takes part as NaN,
+    // which compares false both ways; four scores per shared-memory read
+    sm.S[tid] = elig ? S : __int_as_float(0x7fc00000);
+    sm.par[tid] = par;
     __syncthreads();
-    // rank among eligible nodes by (S descending, index ascending)
     int rank = 0;
     if (elig) {
-        for (int j = 0; j < n; ++j)
-            rank += (s_elig[j] && (s_S[j] > S || (s_S[j] == S && j < tid)));
+        const float4* S4 = reinterpret_cast<const float4*>(sm.S);
+        for (int j = 0; j < n; j += 4) {               // (entries past n belong to threads that are not eligible)
+            const float4 v = S4[j >> 2];
+            rank += (v.x > S || (v.x == S && j < tid)) + (v.y > S || (v.y == S && j + 1 < tid)) +
+                    (v.z > S || (v.z == S && j + 2 < tid)) + (v.w > S || (v.w == S && j + 3 < tid));
+        }
     }
     const bool keep = elig && rank < (p.n_override ? p.n_override[b] : np);
     // compaction: ballot inside the warp, prefix over the four warps
     const unsigned int bal = __ballot_sync(HS_FULL_MASK, keep);
-    __syncthreads();                       // s_warp is reused
-    if (lane == 0) s_warp[warp] = __popc(bal);
+    if (lane == 0) sm.warp[warp] = __popc(bal);
     __syncthreads();
     int before = __popc(bal & ((1u << lane) - 1u));
-    for (int w = 0; w < warp; ++w) before += s_warp[w];
-    const int n_keep = s_warp[0] + s_warp[1] + s_warp[2] + s_warp[3];
-    s_new[tid] = keep ? before : -1;
-    __syncthreads();
+    for (int w = 0; w < warp; ++w) before += sm.warp[w];
+    const int n_keep = sm.warp[0] + sm.warp[1] + sm.warp[2] + sm.warp[3];
+    sm.nw[tid] = keep ? before : -1;
+    const int off = offset_of(n_keep);
+    __syncthreads();                       // sm.nw is complete
     if (keep) {
         const int k = off + before;
         unsigned long long m0 = 0ull, m1 = 0ull;
         int a = tid;
         for (int step = 0; step <= HS_MAX_NODES && a >= 0; ++step) {   // walk to the root
-            int na = s_new[a];
+            int na = sm.nw[a];
             if (na >= 0) {
                 if (na < 64) m0 |= 1ull << na; else m1 |= 1ull << (na - 64);
             }
-            a = s_par[a];
+            a = sm.par[a];
         }
         p.out.keep_idx[k] = tid;
-        p.out.new_parent[k] = par >= 0 ? s_new[par] : -1;
+        p.out.new_parent[k] = par >= 0 ? sm.nw[par] : -1;
         p.out.new_depth[k] = dep;
         p.out.keep_rank[k] = rank;
         p.out.anc_mask[2 * (size_t)k] = m0;
@@ -272,6 +263,134 @@ __global__ void __launch_bounds__(HS_MAX_NODES) stratify_prune_kernel(const Prun
         if (b == p.batch - 1) p.out.keep_off[p.batch] = off + n_keep;
         p.out.status[b] = status;
     }
+}
+
+__global__ void __launch_bounds__(HS_MAX_NODES) stratify_prune_kernel(const PruneParams p) {
+    __shared__ PruneSmem sm;
+    const int tid = threadIdx.x;
+    const int b = blockIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();                            // scores and Phi(P*) come from the kernel ahead in the stream
+    const int base = p.node_off[b];
+    const int n = min(p.node_off[b + 1] - base, HS_MAX_NODES);
+    const int status = p.qstatus[b];
+    int dep = 0, par = -1;
+    float S = 0.f;
+    if (tid < n && status == 0) {
+        dep = p.depth[base + tid];
+        par = p.parent[base + tid];
+        S = p.score[base + tid];
+    }
+    prune_cta(p, b, n, status, p.phi_star[b], dep, par, S, sm, [&](int) {
+        // offset of this sequence in the compacted arrays: the kept counts of the sequences ahead
+        int part = 0;
+        if (p.counted) {
+            for (int bb = tid; bb < b; bb += HS_MAX_NODES) part += p.out.n_keep[bb];
+        } else {
+            for (int bb = tid; bb < b; bb += HS_MAX_NODES) part += kept_count(p, bb);
+        }
+        return cta_sum(part, sm);
+    });
+}
+
+// ---- tree stage and pruning in one launch ---------------------------------------------------------------------
+struct TreePruneParams {
+    // the tree stage's view (the names tree_stage_cta expects)
+    const void* logits;
+    int64_t row_stride;
+    int vocab, is_bf16, prefetch;
+    const int* node_off;
+    const int* parent;
+    const int* token;
+    hs_quant_out out;
+    int d_base, phi_mode, pstar_mode, entropy_mode;
+    PruneParams pr;
+    int* flags;       // [B] kept count + 1 of a sequence once its CTA knows it (zero between launches)
+    int* done;        // CTAs that have read the counts ahead of theirs
+    int* err;         // sticky device error word (a bounded wait that expired)
+};
+
+// One CTA per sequence: the tree stage, then - from shared memory and registers, without a round trip through the
+// quantify outputs - bin, d', N', reranking, compaction and masks.  The offset of a sequence in the compacted arrays
+// needs the kept counts of the sequences ahead, which other CTAs of this launch compute: every CTA publishes its
+// count (release) and reads the counts ahead of it (acquire, bounded wait).  CTAs are started in index order and a
+// CTA only waits for lower indices, so a waiting CTA never keeps the one it waits for from starting.  The CTA that
+// is last to finish its reads puts flags and counter back to zero.
+__global__ void __launch_bounds__(HS_MAX_NODES) tree_prune_kernel(const __grid_constant__ TreePruneParams p) {
+    __shared__ TreeStageSmem tsm;
+    __shared__ PruneSmem sm;
+    const int tid = threadIdx.x;
+    const int b = blockIdx.x;
+    pdl_launch_dependents();
+    const TreeStageResult t = tree_stage_cta(p, b, tsm);
+    __syncthreads();                                   // tsm.phi_star
+    const int n = min(max(t.n, 0), HS_MAX_NODES);
+    const int status = t.bad ? HS_ERR_BAD_TREE : HS_OK;
+    prune_cta(p.pr, b, n, status, t.bad ? 0.f : tsm.phi_star, t.dep, t.bad ? -1 : t.par, t.S, sm, [&](int n_keep) {
+        if (p.pr.batch == 1) return 0;
+        if (tid == 0) st_release_gpu(&p.flags[b], n_keep + 1);
+        int part = 0;
+        const unsigned long long t0 = global_timer_ns();
+        for (int bb = tid; bb < b; bb += HS_MAX_NODES) {
+            int v = ld_acquire_gpu(&p.flags[bb]);
+            while (v == 0) {
+                if (global_timer_ns() - t0 > 2000000000ull) { atomicExch(p.err, HS_ERR_TIMEOUT); v = 1; break; }
+                __nanosleep(64);
+                v = ld_acquire_gpu(&p.flags[bb]);
+            }
+            part += v - 1;
+        }
+        const int off = cta_sum(part, sm);             // (its barriers order every thread's reads before the arrival)
+        if (tid == 0) {
+            int old;
+            asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(old) : "l"(p.done) : "memory");
+            if (old == p.pr.batch - 1) {               // every CTA has read what it needs
+                for (int bb = 0; bb < p.pr.batch; ++bb) p.flags[bb] = 0;
+                *p.done = 0;
+            }
+        }
+        return off;
+    });
+}
+
+hs_status hs_launch_tree_prune(hs_ctx* ctx, const hs_tree_batch* tree, const void* logits, hs_dtype dtype,
+                               int64_t row_stride, int32_t vocab, const hs_policy* policy, const hs_quant_out* quant,
+                               const hs_pruned_tree* out, cudaStream_t stream) {
+    TreePruneParams p;
+    p.logits = logits;
+    p.row_stride = row_stride;
+    p.vocab = vocab;
+    p.is_bf16 = dtype == HS_BF16;
+    p.prefetch = (ctx->prefetch & HS_PREFETCH_LOGITS) != 0;
+    p.node_off = tree->node_off;
+    p.parent = tree->parent;
+    p.token = tree->token;
+    p.out = *quant;
+    p.d_base = policy->d_base;
+    p.phi_mode = policy->phi_mode;
+    p.pstar_mode = policy->pstar_mode;
+    p.entropy_mode = policy->entropy_mode;
+    PruneParams& q = p.pr;
+    q.batch = tree->batch;
+    q.node_off = tree->node_off;
+    q.parent = tree->parent;
+    q.score = quant->score;
+    q.phi_star = quant->phi_star;
+    q.depth = quant->depth;
+    q.qstatus = quant->status;
+    q.out = *out;
+    for (int i = 0; i < 7; ++i) q.th[i] = policy->thresholds[i];
+    q.d_base = policy->d_base;
+    q.alpha = policy->alpha;
+    q.n_default = policy->n_default;
+    for (int i = 0; i < 3; ++i) q.gamma_pct[i] = policy->gamma_pct[i];
+    q.n_override = nullptr; q.base = nullptr; q.room = nullptr; q.slo_class = nullptr; q.budget = 0;
+    q.counted = 0;
+    p.flags = ctx->counters + HS_CNT_PRUNE_FLAG;
+    p.done = ctx->counters + HS_CNT_PRUNE_DONE;
+    p.err = ctx->counters + HS_CNT_ERROR;
+    return hs_launch(tree_prune_kernel, dim3(q.batch), dim3(HS_MAX_NODES), 0, stream, ctx->pdl, dim3(1, 1, 1), p) ==
+                   cudaSuccess ? HS_OK : HS_ERR_CUDA;
 }
 
 hs_status hs_launch_stratify_prune(hs_ctx* ctx, const hs_tree_batch* tree, const hs_quant_out* quant,

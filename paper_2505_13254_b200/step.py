@@ -97,9 +97,18 @@ class VerifyStep:
                                  target_layout=hb.HS_ROWS_ORIGINAL, seed=db.seed, offset=db.offset,
                                  path_cap=self.accept.path_cap, out=self.accept)
 
-    def run(self, db: DeviceBatch):
-        self.quantify(db)
-        self.prune(db)
+    def quantify_prune(self, db: DeviceBatch):
+        return hb.hs_entropy_quantify_prune(self.ctx, db.tree, db.draft, self.policy, out=self.quant,
+                                            pruned_out=self.pruned)
+
+    def run(self, db: DeviceBatch, fused: bool = True):
+        """One verification step.  `fused`: entropy pass, tree scores and pruning as one call of two launches
+        (hs_entropy_quantify_prune) instead of two calls of three."""
+        if fused:
+            self.quantify_prune(db)
+        else:
+            self.quantify(db)
+            self.prune(db)
         if db.q is not None:
             self.attention(db)
         self.accept_path(db)

@@ -314,3 +314,35 @@ def test_every_bin_occurs_and_matches(ctx):
         if len(bins) == 8:
             break
     assert bins == set(range(8))
+
+
+# ---- the fused call (entropy pass, then tree scores + pruning in one kernel) against the two separate calls -------
+
+@pytest.mark.parametrize("batch,seed", [(1, 2600), (7, 2601), (40, 2602), (150, 2603)])
+def test_fused_quantify_prune_equals_the_two_calls(ctx, batch, seed):
+    """The CTAs of the fused kernel hand their kept counts to one another (the offsets of the compacted arrays); with
+    150 sequences more CTAs run than one wave of the small-batch path covers.  Twice in a row: the hand-over flags
+    have put themselves back."""
+    cfg = synth.CONFIGS["c4_ragged"].scaled(batch=batch, vocab=4096, n_nodes=(3, 60))
+    policy = pu.policy_for(cfg, "c4_ragged")
+    batch_np = synth.make_batch(cfg, seed, with_attention=False)
+    db = gstep.upload(batch_np)
+    two = gstep.VerifyStep(ctx, db, policy)
+    two.quantify(db)
+    two.prune(db)
+    one = gstep.VerifyStep(ctx, db, policy)
+    for rep in range(2):
+        for t in (one.pruned.keep_idx, one.pruned.keep_off, one.pruned.n_keep, one.quant.phi):
+            t.fill_(-7)
+        one.quantify_prune(db)
+        torch.cuda.synchronize()
+        for name in ("row_max", "row_lse", "h_full", "i_topk", "topk_idx", "logc", "score", "phi", "depth", "pstar_node",
+                     "phi_star", "status"):
+            assert torch.equal(getattr(one.quant, name), getattr(two.quant, name)), name
+        total = int(two.pruned.keep_off[-1])
+        assert torch.equal(one.pruned.keep_off, two.pruned.keep_off) and torch.equal(one.pruned.n_keep, two.pruned.n_keep)
+        for name in ("keep_idx", "new_parent", "new_depth", "keep_rank", "anc_mask"):
+            assert torch.equal(getattr(one.pruned, name)[:total], getattr(two.pruned, name)[:total]), name
+        for name in ("bin", "d_prime", "n_prime", "status"):
+            assert torch.equal(getattr(one.pruned, name), getattr(two.pruned, name)), name
+    assert hb.hs_device_error(ctx) == 0
