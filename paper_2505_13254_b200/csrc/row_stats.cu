@@ -302,7 +302,11 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
     }
 
     // ---- consumers -------------------------------------------------------------------------------------------------
-    pdl_wait();                    // partials, counters and outputs may still be in use by the kernel ahead
+    // Partials, counters and outputs may still be in use by the kernel ahead: nothing is written before the wait.
+    // Reading the logits and reducing them in registers and shared memory needs no wait if the caller vouches that
+    // they were complete before the call (prefetch): then the wait comes at the end of the first segment.
+    bool waited = false;
+    if (!p.prefetch) { pdl_wait(); waited = true; }
     const int K = p.K;
     const unsigned int ninf = BF16 ? 0xff80ff80u : 0xff800000u;
     int cslot = 0;                 // slot of the next item and the parity of its `full` barrier (the producer fills
@@ -519,6 +523,7 @@ __global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const Qu
         if (ncand <= CAND_CAP) rank_select_warps(s_list, ncand, K, top, warp, lane, NW);
         else topk_by_rounds<BF16>(rowp, sv0, sv1, p.vocab, K, top, s_red, tid, QS_CONSUMERS, 1);   // heavy ties
         bar_sync(1, QS_CONSUMERS);                    // the Top-K is complete; s_list and s_cnt are free again
+        if (!waited) { pdl_wait(); waited = true; }   // from here on the segment's results go to global memory
         int c_first, nseg;
         shares_of_row(p, row, c_first, nseg);
         if (warp == 0) {
