@@ -281,7 +281,7 @@ def main():
     sampler = ClockSampler(local) if rank == 0 else None
     ms = timed_replays(lambda db: st.run(db), args.steps)
     # ---- per-call durations: each call alone, back to back over the rotating inputs ------------------------
-    calls = ("quantify", "prune", "attention", "accept_path")
+    calls = ("quantify", "prune", "quantify_prune", "attention", "accept_path")
     call_us = {c: 1e3 * timed_replays(getattr(st, c), args.steps) / args.steps for c in calls}
     st.run(sets[0])
     barrier()
@@ -365,7 +365,11 @@ def main():
         "accept_path": {"bytes": accept_bytes, "us": call_us["accept_path"],
                         "launches_per_step": 2 if db0.any_sampling else 1},
         "prune": {"bytes": 0, "us": call_us["prune"], "launches_per_step": 1},
+        # what a step runs in place of the two calls above: the entropy pass, then tree scores + pruning in one kernel
+        "quantify_prune": {"bytes": quant_bytes, "us": call_us["quantify_prune"], "launches_per_step": 2},
     }
+    for name in ("quantify", "prune"):
+        kern[name]["in_step"] = False          # timed alone for comparison; the step makes the fused call
     for k in kern.values():
         k["gbs"] = k["bytes"] / (k["us"] * 1e-6) / 1e9 if k["us"] > 0 else None
         k["frac_of_%s_hbm" % peak_kind] = k["gbs"] / peak if k["gbs"] else None
@@ -386,14 +390,15 @@ def main():
                 "d2h_bytes_per_step": d2h, "ms_per_step": 1e3 * e2e_s / e2e_steps,
                 "how": "every step copies all inputs from pinned host memory and reads its results back; the copies of "
                        "step n + 1 overlap the kernels of step n (two staging buffers, two streams)"},
-        "gpu_launches": (6 if db0.any_sampling else 5) * args.steps,
+        "gpu_launches": (5 if db0.any_sampling else 4) * args.steps,
         "roofline": {"kernel": "quantify_stream_kernel (hs_entropy_quantify: this kernel + the tree stage)", "bound": "hbm",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal": achieved / NOMINAL_HBM_GBS,
                      "peak_kind": peak_kind + " (burst copy figure)", "traffic": traffic,
                      "algorithmic_bytes_per_launch": quant_bytes,
                      "how": "CUDA events around K back-to-back graph-replayed calls of hs_entropy_quantify alone (both of its "
-                            "launches in the duration), inputs rotating"},
+                            "launches in the duration), inputs rotating; with programmatic dependent launch and prefetch "
+                            "allowed, the row pass of one call overlaps the tree stage of the call before it"},
         "calls": kern,
         "device_error_word": dev_err,
     }
