@@ -239,8 +239,11 @@ __device__ __forceinline__ int partial_slot(const QuantParams& p, int row, int c
     return 2 * c + ((long long)row * p.nvec < (long long)c * p.per ? 0 : 1);
 }
 
+// 72 registers per thread (no spills): the 17 warps then leave room in the register file for a CTA of the kernel
+// ahead that is still at work on the same SM (in a decode loop: the CTA that walks the accepted path of the step
+// before), so this kernel's CTA is resident, and its share on chip, before that kernel has ended.
 template <bool BF16>
-__global__ void __launch_bounds__(QS_THREADS, 1) quantify_stream_kernel(const QuantParams p) {
+__global__ void __maxnreg__(72) quantify_stream_kernel(const QuantParams p) {
     constexpr int VE = BF16 ? 8 : 4;
     constexpr int NW = QS_CONSUMERS / 32;
     extern __shared__ __align__(128) unsigned char s_dyn[];
