@@ -53,6 +53,7 @@ struct AcceptParams {
     uint4* partials;      // [2][max_rows][chunks] {key lo, key hi, max, sum}
     int* row_cnt;
     int* seq_cnt;         // [batch] merged target rows of a sequence (zero between launches)
+    int clustered;        // chunk kernel: the chunks of a row form a thread-block cluster and merge through shared memory
     int staged;           // the walk may stage row slices in shared memory by bulk copies (16-byte aligned rows)
     int* err;             // sticky device error word (a bounded wait that expired)
 };
@@ -333,10 +334,14 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 4) accept_rows_kernel(const __
     constexpr int VPT = HS_ROW_VPT;
     __shared__ float s_w[8][2];
     __shared__ unsigned long long s_key[8];
+    __shared__ __align__(16) uint4 s_cl[8];       // clustered launch, first CTA of a row: the chunks' results
     __shared__ int s_flag;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int chunk = blockIdx.x, k = blockIdx.y, which = blockIdx.z;   // which: 0 target, 1 draft
     pdl_launch_dependents();
+    // First half of a cluster barrier: when it completes every CTA of the row's cluster runs, and its shared memory may
+    // be written from outside.  (The CTAs of a cluster take every early exit below together: same row, same sequence.)
+    if (p.clustered) cluster_arrive();
     pdl_wait();                            // the pruned tree and the logits come from upstream
     // sequences that kept nothing (flagged upstream) get their empty result from CTA (0, b, 0)
     if (chunk == 0 && which == 0 && k < p.batch && (p.pr.n_keep[k] <= 0 || p.pr.status[k] != 0)) {
@@ -422,6 +427,7 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 4) accept_rows_kernel(const __
     }
     if (lane == 0) s_key[warp] = key;
     __syncthreads();
+    if (p.clustered) cluster_wait();
     if (tid == 0) {
         unsigned long long best = s_key[0];
         for (int w = 1; w < 8; ++w) best = s_key[w] > best ? s_key[w] : best;
@@ -432,24 +438,38 @@ __global__ void __launch_bounds__(HS_ROW_THREADS, 4) accept_rows_kernel(const __
             for (int w = 0; w < 8; ++w)
                 S += (s_w[w][0] == -CUDART_INF_F) ? 0.f : s_w[w][1] * ex2a((s_w[w][0] - M) * invT);
         }
-        p.partials[((size_t)which * p.part_rows + k) * p.chunks + chunk] =
-            make_uint4((unsigned int)best, (unsigned int)(best >> 32), __float_as_uint(M), __float_as_uint(S));
-        // one release-acquire arrival at device scope: this thread's partial is visible to whoever arrives last,
-        // and the last one (then, behind the barrier below, its whole CTA) sees all of them
-        int* cnt = &p.row_cnt[which * HS_MAX_ROWS + k];
-        int old;
-        asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(old) : "l"(cnt) : "memory");
-        s_flag = (old == p.chunks - 1);
-        if (s_flag) *cnt = 0;
+        if (p.clustered) {
+            // the chunk's result goes into slot `chunk` of the first CTA of the row's cluster (posted stores through
+            // distributed shared memory; the cluster barrier below makes them visible there)
+            const unsigned int dst = cluster_map_addr(smem_u32(&s_cl[chunk]), 0);
+            asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"((unsigned int)best),
+                         "r"((unsigned int)(best >> 32)), "r"(__float_as_uint(M)), "r"(__float_as_uint(S)) : "memory");
+            s_flag = (chunk == 0);
+        } else {
+            p.partials[((size_t)which * p.part_rows + k) * p.chunks + chunk] =
+                make_uint4((unsigned int)best, (unsigned int)(best >> 32), __float_as_uint(M), __float_as_uint(S));
+            // one release-acquire arrival at device scope: this thread's partial is visible to whoever arrives last,
+            // and the last one (then, behind the barrier below, its whole CTA) sees all of them
+            int* cnt = &p.row_cnt[which * HS_MAX_ROWS + k];
+            int old;
+            asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(old) : "l"(cnt) : "memory");
+            s_flag = (old == p.chunks - 1);
+            if (s_flag) *cnt = 0;
+        }
     }
-    __syncthreads();
+    if (p.clustered) {
+        cluster_arrive();
+        cluster_wait();
+    } else {
+        __syncthreads();
+    }
     if (!s_flag) return;
     if (warp == 0) {
-    // last chunk of the row: merge (chunks <= 32, one lane per chunk)
+    // the CTA that merges the row (chunks <= 32, one lane per chunk)
     unsigned long long ck = 0ull;
     float cm = -CUDART_INF_F, cs = 0.f;
     if (lane < p.chunks) {
-        uint4 q = __ldcg(&p.partials[((size_t)which * p.part_rows + k) * p.chunks + lane]);
+        const uint4 q = p.clustered ? s_cl[lane] : __ldcg(&p.partials[((size_t)which * p.part_rows + k) * p.chunks + lane]);
         ck = ((unsigned long long)q.y << 32) | q.x;
         cm = __uint_as_float(q.z);
         cs = __uint_as_float(q.w);
@@ -1284,6 +1304,7 @@ hs_status hs_launch_accept(hs_ctx* ctx, const hs_tree_batch* tree, const hs_prun
     p.seq_cnt = ctx->counters + HS_CNT_ACC_SEQ;
     p.err = ctx->counters + HS_CNT_ERROR;
     p.staged = 0;
+    p.clustered = 0;
     // without draft logits every sequence must be greedy: no draft rows to scan and no sampling walk
     cudaError_t e;
     const bool streamed = ctx->row_pass == HS_ROW_PASS_STREAM ||
@@ -1300,10 +1321,16 @@ hs_status hs_launch_accept(hs_ctx* ctx, const hs_tree_batch* tree, const hs_prun
             ? hs_launch(accept_stream_kernel<true>, dim3(ctx->sm_count), dim3(AS_THREADS), AS_SMEM_BYTES, stream, ctx->pdl, dim3(1, 1, 1), p)
             : hs_launch(accept_stream_kernel<false>, dim3(ctx->sm_count), dim3(AS_THREADS), AS_SMEM_BYTES, stream, ctx->pdl, dim3(1, 1, 1), p);
     } else {
-        dim3 grid(p.chunks, rows, p.have_draft ? 2 : 1);
+        // up to eight chunks per row (the portable cluster size): the CTAs of a row are one cluster, and the row is
+        // merged in the shared memory of its first CTA instead of through partials and a counter in global memory
+        // - while the whole grid is resident at once (four CTAs per SM): with more CTAs the clusters wait for eight free
+        // slots in one GPC and the pass gets slower than with independent CTAs
+        p.clustered = p.chunks > 1 && p.chunks <= 8 &&
+                      (size_t)p.chunks * rows * (p.have_draft ? 2 : 1) * 2 <= (size_t)7 * ctx->sm_count;
+        dim3 grid(p.chunks, rows, p.have_draft ? 2 : 1), cl(p.clustered ? p.chunks : 1, 1, 1);
         e = dtype == HS_BF16
-            ? hs_launch(accept_rows_kernel<true>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p)
-            : hs_launch(accept_rows_kernel<false>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, dim3(1, 1, 1), p);
+            ? hs_launch(accept_rows_kernel<true>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, cl, p)
+            : hs_launch(accept_rows_kernel<false>, grid, dim3(HS_ROW_THREADS), 0, stream, ctx->pdl, cl, p);
     }
     if (e != cudaSuccess) return HS_ERR_CUDA;
     if (!p.have_draft) return HS_OK;
