@@ -1152,9 +1152,15 @@ accept_walk_kernel(const AcceptParams p) {
     __shared__ int s_par[HS_MAX_NODES], s_tok[HS_MAX_NODES], s_orig[HS_MAX_NODES];
     __shared__ float s_pt[HS_MAX_NODES], s_qt[HS_MAX_NODES], s_u[HS_MAX_NODES];
     __shared__ float2 s_pms[HS_MAX_NODES];
+    // Also per node: its first (lowest-index) kept child and whether that child, tested first (residual = p), is
+    // accepted - the common step of the walk then costs two shared-memory reads.
+    __shared__ int s_first[HS_MAX_NODES];
+    __shared__ unsigned char s_acc0[HS_MAX_NODES];
     const float T = p.temperature[b];
     const float invT = LOG2E / T;
     const int nkc = min(nk, HS_MAX_NODES);
+    for (int j = tid; j < nkc; j += WALK_THREADS) s_first[j] = 0x7fffffff;
+    __syncthreads();
     for (int j = tid; j < nkc; j += WALK_THREADS) {
         const int par = p.pr.new_parent[koff + j];
         const int orig = p.pr.keep_idx[koff + j];
@@ -1172,7 +1178,13 @@ accept_walk_kernel(const AcceptParams p) {
             qt = exp2f((fmaxf(load_logit(qrow, p.is_bf16, tok), -1e30f) - qms.x) * invT) * (1.f / qms.y);
         }
         s_pt[j] = pt; s_qt[j] = qt;
-        s_u[j] = p.uniforms ? p.uniforms[nbase + orig] : philox_uniform(p.seed, p.offset, b, orig, 0);
+        const float u = p.uniforms ? p.uniforms[nbase + orig] : philox_uniform(p.seed, p.offset, b, orig, 0);
+        s_u[j] = u;
+        // (the same expressions as in the sibling loop below with c = 0, W = 1: the same decision, bit for bit)
+        const float r0 = fmaxf(pt - 0.f * qt, 0.f) / 1.f;
+        const float a0 = qt > 0.f ? fminf(1.f, r0 / qt) : 1.f;
+        s_acc0[j] = (par >= 0 && par < j && u < a0) ? 1 : 0;
+        if (par >= 0 && par < j) atomicMin(&s_first[par], j);
     }
     __syncthreads();
     int cur = 0, len = 0, bonus = -1;
@@ -1181,6 +1193,15 @@ accept_walk_kernel(const AcceptParams p) {
             if (rank == 0 && tid == 0 && len < cap) {
                 p.out.path_compact[b * cap + len] = cur;
                 p.out.path_nodes[b * cap + len] = s_orig[cur];
+            }
+            {
+                const int j1 = s_first[cur];
+                if (j1 != 0x7fffffff && s_acc0[j1]) {            // the first child is accepted: no residual is needed
+                    if (rank == 0 && tid == 0 && len < cap) p.out.path_tokens[b * cap + len] = s_tok[j1];
+                    cur = j1;
+                    ++len;
+                    continue;
+                }
             }
             const int trow = p.target_layout == HS_ROWS_ORIGINAL ? nbase + s_orig[cur] : koff + cur;
             const int drow = nbase + s_orig[cur];
