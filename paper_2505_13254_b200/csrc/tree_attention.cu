@@ -397,7 +397,11 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm
             mxb = max3(mxb, __uint_as_float(sr[32 + c]), __uint_as_float(sr[33 + c]));
         }
         const float mx = fmaxf(mxa, mxb) * p.scale_log2;
-        const float mnew = fmaxf(mrun, mx);
+        // The reference the exponents are taken against only follows the row's maximum when that has grown by more
+        // than 8 (a factor 256): until then P <= 256 instead of <= 1, which costs no precision (fp32 sums, bf16 keeps
+        // its relative error, the final O / l is the same quotient), and O is rescaled a few times per row instead of
+        // whenever any row of the warp sees a new maximum.
+        const float mnew = (mx > mrun + 8.f || mrun == -CUDART_INF_F) ? fmaxf(mrun, mx) : mrun;
         const float muse = (mnew == -CUDART_INF_F) ? 0.f : mnew;
         const float corr = ex2_approx(mrun - muse);          // 1 when the maximum did not grow, 0 at the stream's first tile
         mrun = mnew;
