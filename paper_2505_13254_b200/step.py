@@ -86,8 +86,12 @@ class VerifyStep:
         return hb.hs_stratify_prune(self.ctx, db.tree, self.quant, self.policy, out=self.pruned)
 
     def attention(self, db: DeviceBatch, max_nodes: Optional[int] = None):
+        # The launch is sized by an upper bound of the kept nodes per sequence: what the policy keeps at most of one
+        # tree (hs_stratify_prune; a budgeted pruning may keep more: pass the drafted tree size then).
+        if max_nodes is None:
+            max_nodes = keep_bound(self.policy, db.max_nodes)
         return hb.hs_tree_verify_attention(self.ctx, self.pruned, db.q, db.k_tree, db.v_tree, db.k_cache, db.v_cache,
-                                           db.kv_off, batch=db.tree.batch, max_nodes=max_nodes or db.max_nodes,
+                                           db.kv_off, batch=db.tree.batch, max_nodes=max_nodes,
                                            max_kv_len=db.max_kv_len, layout=hb.HS_ROWS_ORIGINAL,
                                            node_off=db.tree.node_off, out=self.attn_out, lse_out=self.attn_lse)
 
@@ -149,6 +153,15 @@ class GraphedStep:
     def replay(self) -> VerifyStep:
         self.graph.replay()
         return self.step
+
+
+def keep_bound(policy: dict, max_nodes: int) -> int:
+    """Most nodes hs_stratify_prune keeps of one tree: the largest N' of the policy's regimes (Sec. 4.3), capped by
+    the drafted tree size."""
+    n = policy["n_default"]
+    for i in range(3):
+        n = max(n, (policy["gamma_pct"][i] * policy["n_default"] + 50) // 100 + policy["alpha"] - i)
+    return max(1, min(max_nodes, n))
 
 
 def regime_bounds(policy: dict, max_nodes: int):
