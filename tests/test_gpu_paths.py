@@ -318,12 +318,13 @@ def test_every_bin_occurs_and_matches(ctx):
 
 # ---- the fused call (entropy pass, then tree scores + pruning in one kernel) against the two separate calls -------
 
-@pytest.mark.parametrize("batch,seed", [(1, 2600), (7, 2601), (40, 2602), (150, 2603)])
-def test_fused_quantify_prune_equals_the_two_calls(ctx, batch, seed):
-    """The CTAs of the fused kernel hand their kept counts to one another (the offsets of the compacted arrays); with
-    150 sequences more CTAs run than one wave of the small-batch path covers.  Twice in a row: the hand-over flags
-    have put themselves back."""
-    cfg = synth.CONFIGS["c4_ragged"].scaled(batch=batch, vocab=4096, n_nodes=(3, 60))
+@pytest.mark.parametrize("batch,seed,nodes", [(1, 2600, (3, 60)), (7, 2601, (3, 60)), (40, 2602, (3, 60)),
+                                              (150, 2603, (3, 60)), (3000, 2604, (2, 6))])
+def test_fused_quantify_prune_equals_the_two_calls(ctx, batch, seed, nodes):
+    """The CTAs of the fused kernel hand their kept counts to one another (the offsets of the compacted arrays).
+    With 3000 sequences there are more CTAs than the device holds at once: a CTA only waits for lower-numbered
+    ones, which were started before it.  Twice in a row: the hand-over flags have put themselves back."""
+    cfg = synth.CONFIGS["c4_ragged"].scaled(batch=batch, vocab=4096 if batch < 1000 else 512, n_nodes=nodes)
     policy = pu.policy_for(cfg, "c4_ragged")
     batch_np = synth.make_batch(cfg, seed, with_attention=False)
     db = gstep.upload(batch_np)
