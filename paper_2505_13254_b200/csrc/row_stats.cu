@@ -48,6 +48,7 @@ struct QuantParams {
     int split;       // stream kernel: shares per row (row-split geometry), 0 = byte-balanced stream
     int extra;       // stream kernel, row split: the first `extra` rows have one share more
     int nslots;      // stream kernel: item slots in shared memory
+    int clustered;   // stream kernel, row split: the shares of a row are one thread-block cluster and merge in shared memory
     int rows;
     int batch;
     const int* node_off;
@@ -256,6 +257,8 @@ __global__ void __maxnreg__(72) quantify_stream_kernel(const QuantParams p) {
     __shared__ float s_wstat[2][NW][3];
     __shared__ int s_cnt;
     __shared__ int s_flag;
+    __shared__ unsigned long long s_ck[8][HS_MAX_TOPK];   // clustered launch, first CTA of a row: the shares' Top-K keys
+    __shared__ __align__(16) float4 s_cs[8];               //   and their {max, sum e, sum x e}
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned int slots0 = (smem_u32(s_dyn) + 127u) & ~127u;
@@ -275,6 +278,10 @@ __global__ void __maxnreg__(72) quantify_stream_kernel(const QuantParams p) {
     }
     __syncthreads();
     pdl_launch_dependents();
+    // Clustered launch: first half of a cluster barrier - when it completes every CTA of the row's cluster runs and
+    // its shared memory may be written from outside.  Every thread of the CTA, the producer warp included, takes part
+    // in the two barrier phases of the launch.
+    if (p.clustered) cluster_arrive();
 
     if (warp == NW) {
         // ---- producer: one lane walks the share item by item ----------------------------------------------------
@@ -300,6 +307,12 @@ __global__ void __maxnreg__(72) quantify_stream_kernel(const QuantParams p) {
                 ++it;
                 if (++slot == nslots) { slot = 0; epar ^= 1u; }
             }
+        }
+        if (p.clustered) {
+            __syncwarp();
+            cluster_wait();
+            cluster_arrive();
+            cluster_wait();
         }
         return;
     }
@@ -527,6 +540,7 @@ __global__ void __maxnreg__(72) quantify_stream_kernel(const QuantParams p) {
         else topk_by_rounds<BF16>(rowp, sv0, sv1, p.vocab, K, top, s_red, tid, QS_CONSUMERS, 1);   // heavy ties
         bar_sync(1, QS_CONSUMERS);                    // the Top-K is complete; s_list and s_cnt are free again
         if (!waited) { pdl_wait(); waited = true; }   // from here on the segment's results go to global memory
+        if (p.clustered) cluster_wait();              // (the arrival at the start: every CTA of the cluster runs)
         int c_first, nseg;
         shares_of_row(p, row, c_first, nseg);
         if (warp == 0) {
@@ -545,6 +559,20 @@ __global__ void __maxnreg__(72) quantify_stream_kernel(const QuantParams p) {
             if (nseg == 1) {
                 // the whole row lay in this share: the other warps are already on their way to the next segment
                 finalize_row(p, row, M, St, Ut, top, lane);
+            } else if (p.clustered) {
+                // this share's partial goes into slot `part` of the first CTA of the row's cluster (posted stores
+                // through distributed shared memory; the cluster barrier below makes them visible there)
+                const int part = blockIdx.x - c_first;
+                if (lane < HS_MAX_TOPK) {
+                    const unsigned int dst = cluster_map_addr(smem_u32(&s_ck[part][lane]), 0);
+                    asm volatile("st.shared::cluster.b64 [%0], %1;" ::"r"(dst), "l"((lane < K) ? top[lane] : 0ull) : "memory");
+                }
+                if (lane == 0) {
+                    const unsigned int dst = cluster_map_addr(smem_u32(&s_cs[part]), 0);
+                    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(__float_as_uint(M)),
+                                 "r"(__float_as_uint(St)), "r"(__float_as_uint(Ut)), "r"(0u) : "memory");
+                    s_flag = (part == 0);
+                }
             } else {
                 const int ps = partial_slot(p, row, blockIdx.x);
                 if (lane == 0) p.part_stats[ps] = make_float4(M, St, Ut, 0.f);
@@ -562,13 +590,23 @@ __global__ void __maxnreg__(72) quantify_stream_kernel(const QuantParams p) {
             }
         }
         if (nseg > 1) {
-            bar_sync(1, QS_CONSUMERS);                // s_flag
+            if (p.clustered) {
+                cluster_arrive();                     // (second phase: the stores above are released, and acquired below)
+                cluster_wait();
+            } else {
+                bar_sync(1, QS_CONSUMERS);            // s_flag
+            }
             if (s_flag) {
-                // ---- the last share of a split row merges the row's partials ---------------------------------------
+                // ---- the last share of a split row (clustered: the first CTA of its cluster) merges the partials ----
                 if (tid < HS_MAX_TOPK) top[tid] = 0ull;
                 float4 stv = make_float4(-CUDART_INF_F, 0.f, 0.f, 0.f);       // (warp 0: requested with the keys)
-                if (warp == 0 && lane < nseg) stv = __ldcg(&p.part_stats[partial_slot(p, row, c_first + lane)]);
+                if (warp == 0 && lane < nseg)
+                    stv = p.clustered ? s_cs[lane] : __ldcg(&p.part_stats[partial_slot(p, row, c_first + lane)]);
                 for (int t = tid; t < nseg * HS_MAX_TOPK; t += QS_CONSUMERS) {
+                    if (p.clustered) {
+                        s_list[t] = s_ck[t / HS_MAX_TOPK][t % HS_MAX_TOPK];
+                        continue;
+                    }
                     const int ps = partial_slot(p, row, c_first + t / HS_MAX_TOPK);
                     s_list[t] = __ldcg(&p.part_keys[(size_t)ps * HS_MAX_TOPK + (t % HS_MAX_TOPK)]);
                 }
@@ -586,6 +624,11 @@ __global__ void __maxnreg__(72) quantify_stream_kernel(const QuantParams p) {
         }
         ++seg;
         g = row_g0 + sv1;
+    }
+    if (p.clustered && seg == 0) {                    // (a CTA without a segment still owes the cluster its two phases)
+        cluster_wait();
+        cluster_arrive();
+        cluster_wait();
     }
 }
 
@@ -611,6 +654,7 @@ static void fill_common(QuantParams& p, const hs_tree_batch* tree, const void* l
     p.split = 0;
     p.extra = 0;
     p.nslots = QS_SLOTS;
+    p.clustered = 0;
     p.rows = tree->n_nodes_total;
     p.batch = tree->batch;
     p.node_off = tree->node_off;
@@ -637,12 +681,27 @@ static void quantify_geometry(int rows, int nvec, int sm_count, QuantParams& p, 
     while (S > 1 && (S + 1 > QS_MAX_SEGS || nvec / (S + 1) < 256)) --S;      // parts of at least 4 KiB
     const int extra = (S >= 1 && S + 1 <= QS_MAX_SEGS && nvec / (S + 1) >= 256) ? min(rows, sm_count - rows * S) : 0;
     const int pv_max = S >= 1 ? (nvec + S - 1) / S : 0;
+    // With at most half as many rows as SMs every row is cut into the same number of parts (at most eight, the portable
+    // cluster size): the CTAs of a row are one thread-block cluster and merge the row in the shared memory of its first
+    // CTA.  (The critical path is the same as with one part more for some rows - the rows with fewer parts - but the
+    // merge costs a cluster barrier instead of partials, an atomic and their read-back through global memory.)
+    int Sc = rows <= sm_count / 2 ? (sm_count / rows < 8 ? sm_count / rows : 8) : 0;
+    while (Sc > 1 && nvec / Sc < 256) --Sc;
+    const int pv_c = Sc >= 2 ? (nvec + Sc - 1) / Sc : 0;
+    p.clustered = 0;
     if (rows >= 2 * sm_count) {
         p.split = -1;
         p.extra = sm_count;
         p.per = 0;
         p.nslots = QS_SLOTS;
         nctas = sm_count;
+    } else if (Sc >= 2 && pv_c <= QS_SLOTS * QS_ITEM_VECS) {
+        p.split = Sc;
+        p.extra = 0;
+        p.per = pv_c;
+        p.nslots = (pv_c + QS_ITEM_VECS - 1) / QS_ITEM_VECS;
+        p.clustered = 1;
+        nctas = rows * Sc;
     } else if (S >= 1 && pv_max <= QS_SLOTS * QS_ITEM_VECS) {
         p.split = S;
         p.extra = extra;
@@ -689,8 +748,10 @@ hs_status hs_launch_quantify(hs_ctx* ctx, const hs_tree_batch* tree, const void*
         ctx->quant_ready = true;
     }
     cudaError_t e = dtype == HS_BF16
-        ? hs_launch(quantify_stream_kernel<true>, dim3(nctas), dim3(QS_THREADS), smem, stream, ctx->pdl, dim3(1, 1, 1), p)
-        : hs_launch(quantify_stream_kernel<false>, dim3(nctas), dim3(QS_THREADS), smem, stream, ctx->pdl, dim3(1, 1, 1), p);
+        ? hs_launch(quantify_stream_kernel<true>, dim3(nctas), dim3(QS_THREADS), smem, stream, ctx->pdl,
+                    dim3(p.clustered ? p.split : 1, 1, 1), p)
+        : hs_launch(quantify_stream_kernel<false>, dim3(nctas), dim3(QS_THREADS), smem, stream, ctx->pdl,
+                    dim3(p.clustered ? p.split : 1, 1, 1), p);
     if (e != cudaSuccess) return HS_ERR_CUDA;
     if (!with_tree_stage) return HS_OK;              // (the caller launches the kernel that also prunes)
     e = hs_launch(tree_scores_kernel, dim3(p.batch), dim3(HS_MAX_NODES), 0, stream, ctx->pdl, dim3(1, 1, 1), p);
