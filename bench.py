@@ -449,7 +449,7 @@ def main():
                              "two_phase_us": wall(rs.replay), "one_graph_us": wall(one.replay)}
         line["regime_graphs"] = dict(regimes, how="wall clock per step over back-to-back replays on one input copy (L2-warm); "
                                      "two_phase = quantify + prune, the host reads the kept-node count, then the regime's own "
-                                     "graph of attention + acceptance; one_graph = all calls in one graph sized by the drafted tree")
+                                     "graph of attention + acceptance; one_graph = all calls in one graph sized by the drafted tree (the attention: by the most the policy keeps)")
     if not args.no_cpu_baseline:
         from oracle import step as ostep
         nrep = 5
