@@ -1,13 +1,17 @@
-// hs_accept_path: two launches.
+// hs_accept_path: the row pass (one of two kernels) and, with draft logits, the walk.
 //
 // accept_rows_kernel   vocabulary pass over the target row of every kept node (arg-max with lowest
 //                      index on ties; for sampling sequences also max and sum e^((x-max)/T)) and
 //                      over the draft row of every kept internal node of a sampling sequence.
-//                      Same register-resident 16-byte-load pattern as the entropy pass; the last
-//                      chunk of a row merges the chunk partials.
-//                      Greedy sequences and sequences with deterministic proposals finish here: the CTA
-//                      that merges a sequence's last target row walks its tree (greedy_walk,
-//                      deterministic_walk).
+//                      A CTA per 32 KiB chunk of a row, all 16-byte loads in flight at once (launches
+//                      with few rows); the chunks of a row merge in the shared memory of a thread-block
+//                      cluster, or through partials and an arrival counter where the grid is too large
+//                      for clusters to pay.
+// accept_stream_kernel the same pass for launches with many rows: one persistent CTA per SM, a producer
+//                      warp and a ring of shared-memory slots (see the comment ahead of the kernel).
+//                      Greedy sequences and sequences with deterministic proposals finish in the row
+//                      pass: the CTA that completes a sequence's last target row walks its tree
+//                      (greedy_walk, deterministic_walk).
 // accept_walk_kernel   one thread-block cluster per sequence walks the tree from the root.
 //                      Greedy (temperature 0): follow the child whose token is the arg-max.
 //                      Sampling (Sec. 2.1): test siblings in index order with u < min(1, r/q); the

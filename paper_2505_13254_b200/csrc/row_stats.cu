@@ -11,9 +11,12 @@
 //     re-scan their vectors in shared memory and push candidates; the few candidates are ranked by counting.
 //     A share that ends inside a row leaves a partial {max, sum, sum x e, K keys}; the last CTA of a row to
 //     arrive merges the partials into max, log-sum-exp, Shannon entropy, Top-K and the two Top-K entropies
-//     (Eq. 1 inner sum).  Rows that lie inside one share need no partial and no atomic.
+//     (Eq. 1 inner sum).  Rows that lie inside one share need no partial and no atomic.  With few rows every row
+//     is cut into the same number of shares, which form a thread-block cluster: the partials then go into the
+//     shared memory of the cluster's first CTA instead of through global memory.
 // tree_scores_kernel       One CTA per sequence: path confidence ln V_i (Sec. 2.2), cumulative meta-path
-//     Top-K entropy Phi (Eq. 1) and the operational path P* (Sec. 4.1).
+//     Top-K entropy Phi (Eq. 1) and the operational path P* (Sec. 4.1).  (The fused call launches the kernel
+//     of stratify_prune.cu that runs the same tree stage and then prunes, in its place.)
 //
 // quantify_chunk_kernel (a CTA owns one chunk of one row, registers only) serves the allocation-free entry.
 #include <math_constants.h>

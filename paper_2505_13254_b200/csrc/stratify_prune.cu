@@ -7,6 +7,9 @@
 // every CTA recomputes those counts itself, so no CTA waits for another and the call is one launch.
 // Larger batches: a first launch counts the kept nodes of every sequence once (one warp each), the
 // second sums the counts ahead of its sequence (B integers instead of B trees per CTA).
+//
+// hs_entropy_quantify_prune launches tree_prune_kernel instead: the tree stage (path scores, Phi, P*) and the
+// pruning of a sequence in one CTA; there the kept counts are handed from CTA to CTA (release / acquire flags).
 #include "hs_common.cuh"
 #include "hs_layout.h"
 #include "hs_ptx.cuh"
